@@ -1,0 +1,89 @@
+"""Planted mistakes: each mutant of the oracle source must be caught by at least one pin.
+
+The mistake is planted in a temporary copy of the oracle's C source, on the CPU; the
+pins of test_oracle_pins.py are then re-run against the mutant library."""
+import ctypes
+import os
+import subprocess
+
+import pytest
+
+import oracle
+import test_oracle_pins as pins
+
+MUTANTS = {
+    "scale_dropped": ("s[j] = scale * acc;", "s[j] = acc;"),
+    "not_normalised": ("REAL p = s[j] / denom;", "REAL p = s[j];"),
+    "value_dims_reversed": ("out[d] += p * widen(V[(size_t)j * hd + d]);",
+                            "out[d] += p * widen(V[(size_t)j * hd + (hd - 1 - d)]);"),
+    "query_dims_reversed": ("acc += widen(q[d]) *", "acc += widen(q[hd - 1 - d]) *"),
+    "key_used_as_value": ("out[d] += p * widen(V[", "out[d] += p * widen(K["),
+    "causal_excludes_self": ("Kb, Vb, t + 1, hd", "Kb, Vb, t, hd"),
+    "causal_sees_one_ahead": ("Kb, Vb, t + 1, hd", "Kb, Vb, (t + 2 > T ? T : t + 2), hd"),
+    "decode_drops_last_row": ("int n = len[b];", "int n = len[b] - 1;"),
+    "decode_reads_one_past": ("int n = len[b];", "int n = len[b] + 1;"),
+    "token_excludes_itself": ("int n = appended ? len_old + i + 1 : len_old;",
+                              "int n = appended ? len_old + i : len_old;"),
+    "token_reset_ignored": ("if (do_reset) len[b] = 0;", ";"),
+    "append_ignores_length": ("* cap + (size_t)(len[b] + i)) * hd;", "* cap + (size_t)(i)) * hd;"),
+    "append_no_length_update": ("        len[b] += n_new;", "        ;"),
+    "prefill_ignores_stride": ("(size_t)bh * (size_t)kv_seq_stride * hd;", "(size_t)bh * (size_t)T * hd;"),
+    "heads_swapped_in_decode": ("attend_rows(q + bh * hd, kc + bh * cap * hd,",
+                                "attend_rows(q + ((size_t)b * H + (H - 1 - h)) * hd, kc + bh * cap * hd,"),
+}
+
+PIN_FUNCS = [
+    pins.test_single_row_returns_its_value_exactly,
+    pins.test_equal_keys_give_mean_of_values,
+    pins.test_two_rows_is_a_logistic_blend,
+    pins.test_handmade_scores_one_two_three,
+    pins.test_dominant_key_selects_its_value,
+    lambda: pins.test_probabilities_sum_to_one_and_hull(5),
+    lambda: pins.test_brute_force_tiny(6, 8),
+    pins.test_prefill_matches_library_causal_attention,
+    pins.test_prefill_honours_kv_stride,
+    pins.test_cached_decode_equals_full_recompute,
+    pins.test_block_length_one_is_vanilla_causal_attention,
+    pins.test_ragged_lengths_and_rows_past_len_are_ignored,
+    pins.test_spike_row_at_the_length_boundary,
+    pins.test_append_overflow_and_empty_cache,
+    lambda: pins.test_token_decoder_never_crosses_a_block_boundary(4, 2),
+    pins.test_token_step_equals_attention_over_prefix_plus_same_block_tokens,
+    pins.test_token_attend_only_and_masked_reset,
+]
+
+
+def build_mutant(tmp_path, name, old, new):
+    src = open(os.path.join(os.path.dirname(oracle.__file__), "bt_oracle.c")).read()
+    assert src.count(old) >= 1, f"mutation site for {name} not found"
+    mutated = src.replace(old, new)
+    c = tmp_path / f"{name}.c"
+    c.write_text(mutated)
+    objs = []
+    for real, sfx in (("double", ""), ("float", "_f32")):
+        o = tmp_path / f"{name}{sfx}.o"
+        subprocess.check_call(["gcc", "-O1", "-fopenmp", "-fPIC", "-std=c11", f"-DREAL={real}",
+                               f"-DSUFFIX={sfx}", "-c", str(c), "-o", str(o)])
+        objs.append(str(o))
+    so = tmp_path / f"lib{name}.so"
+    subprocess.check_call(["gcc", "-shared", "-fopenmp", "-o", str(so)] + objs + ["-lm"])
+    return ctypes.CDLL(str(so))
+
+
+@pytest.mark.parametrize("name", sorted(MUTANTS))
+def test_mutant_is_caught(name, tmp_path, monkeypatch):
+    old, new = MUTANTS[name]
+    oracle.lib()  # make sure the real one is built first
+    monkeypatch.setattr(oracle, "_lib", build_mutant(tmp_path, name, old, new))
+    caught = []
+    for f in PIN_FUNCS:
+        try:
+            f()
+        except AssertionError:
+            caught.append(getattr(f, "__name__", "pin"))
+    assert caught, f"no pin noticed the planted mistake '{name}'"
+
+
+def test_unmutated_source_passes_the_same_pins():
+    for f in PIN_FUNCS:
+        f()

@@ -1,0 +1,389 @@
+"""Pins for the CPU oracle: closed forms, invariants the paper fixes, a library routine
+and brute force.  None of these call the CUDA path."""
+import math
+import os
+
+import numpy as np
+import pytest
+import torch
+
+import oracle
+from workloads import gen
+
+HD = 16
+
+
+def bits(x):
+    return gen.f32_to_bf16_bits(np.asarray(x, np.float32))
+
+
+def widen(b):
+    return gen.bf16_bits_to_f32(b).astype(np.float64)
+
+
+def rnd(seed, tid, shape):
+    return gen.normal_bf16_bits(seed, tid, shape)
+
+
+# ---------------------------------------------------------------- closed forms
+
+def test_single_row_returns_its_value_exactly():
+    q, K, V = rnd(1, 0, (HD,)), rnd(1, 1, (1, HD)), rnd(1, 2, (1, HD))
+    out, p = oracle.attend(q, K, V)
+    assert p.tolist() == [1.0]
+    assert np.array_equal(out, widen(V[0]))
+
+
+def test_equal_keys_give_mean_of_values():
+    q = rnd(2, 0, (HD,))
+    K = np.repeat(rnd(2, 1, (1, HD)), 7, axis=0)
+    V = rnd(2, 2, (7, HD))
+    out, p = oracle.attend(q, K, V)
+    np.testing.assert_allclose(p, np.full(7, 1 / 7), rtol=0, atol=1e-15)
+    np.testing.assert_allclose(out, widen(V).mean(0), rtol=0, atol=1e-14)
+
+
+def test_zero_query_gives_mean_of_values():
+    q = np.zeros(HD, np.uint16)
+    K, V = rnd(3, 1, (9, HD)), rnd(3, 2, (9, HD))
+    out, _ = oracle.attend(q, K, V)
+    np.testing.assert_allclose(out, widen(V).mean(0), rtol=0, atol=1e-14)
+
+
+def test_two_rows_is_a_logistic_blend():
+    # with two rows softmax reduces to the logistic function of the score difference
+    q, K, V = rnd(4, 0, (HD,)), rnd(4, 1, (2, HD)), rnd(4, 2, (2, HD))
+    scale = 0.37
+    s = scale * (widen(K) @ widen(q))
+    w0 = 1.0 / (1.0 + math.exp(-(s[0] - s[1])))
+    out, _ = oracle.attend(q, K, V, scale=scale)
+    np.testing.assert_allclose(out, widen(V[1]) + w0 * (widen(V[0]) - widen(V[1])), rtol=0, atol=1e-13)
+
+
+def test_handmade_scores_one_two_three():
+    # q = e0, keys with first coordinate 0, 1, 2 and scale = ln 2  ->  weights 1/7, 2/7, 4/7
+    q = bits([1.0] + [0.0] * (HD - 1))
+    K = np.zeros((3, HD), np.float32)
+    K[:, 0] = [0.0, 1.0, 2.0]
+    K[:, 1] = [5.0, -3.0, 2.0]  # orthogonal to q: must not matter
+    V = np.zeros((3, HD), np.float32)
+    V[:, 0] = [7.0, 14.0, 21.0]
+    V[:, 3] = [1.0, 0.0, 0.0]
+    out, p = oracle.attend(q, bits(K), bits(V), scale=math.log(2.0))
+    np.testing.assert_allclose(p, [1 / 7, 2 / 7, 4 / 7], rtol=0, atol=1e-15)
+    np.testing.assert_allclose(out[0], 1.0 + 4.0 + 12.0, rtol=0, atol=1e-13)
+    np.testing.assert_allclose(out[3], 1 / 7, rtol=0, atol=1e-15)
+
+
+def test_dominant_key_selects_its_value():
+    q = bits(np.full(HD, 4.0))
+    K = rnd(5, 1, (33, HD))
+    V = rnd(5, 2, (33, HD))
+    K[17] = bits(np.full(HD, 16.0))  # score 1024*scale, far above the rest
+    out, p = oracle.attend(q, K, V, scale=1.0)
+    assert p[17] > 1 - 1e-12
+    np.testing.assert_allclose(out, widen(V[17]), rtol=0, atol=1e-9)
+
+
+# ---------------------------------------------------------------- properties
+
+@pytest.mark.parametrize("n", [1, 2, 5, 64, 513])
+def test_probabilities_sum_to_one_and_hull(n):
+    q, K, V = rnd(6, n, (HD,)), rnd(6, 100 + n, (n, HD)), rnd(6, 200 + n, (n, HD))
+    out, p = oracle.attend(q, K, V)
+    assert abs(p.sum() - 1.0) < 1e-12 and (p >= 0).all()
+    Vf = widen(V)
+    assert (out <= Vf.max(0) + 1e-12).all() and (out >= Vf.min(0) - 1e-12).all()
+
+
+def test_permutation_invariance():
+    n = 50
+    q, K, V = rnd(7, 0, (HD,)), rnd(7, 1, (n, HD)), rnd(7, 2, (n, HD))
+    perm = np.random.default_rng(0).permutation(n)
+    a, _ = oracle.attend(q, K, V)
+    b, _ = oracle.attend(q, K[perm], V[perm])
+    np.testing.assert_allclose(a, b, rtol=0, atol=1e-13)
+
+
+def test_log_sum_exp_merge_of_two_halves_equals_whole():
+    # the algebra a split of the row range relies on, checked against the unsplit definition
+    n, cut = 40, 13
+    q, K, V = rnd(8, 0, (HD,)), rnd(8, 1, (n, HD)), rnd(8, 2, (n, HD))
+    scale = oracle.default_scale(HD)
+    whole, _ = oracle.attend(q, K, V)
+    parts = []
+    for sl in (slice(0, cut), slice(cut, n)):
+        o, _ = oracle.attend(q, K[sl], V[sl])
+        s = scale * (widen(K[sl]) @ widen(q))
+        parts.append((o, s.max() + math.log(np.exp(s - s.max()).sum())))
+    (o1, l1), (o2, l2) = parts
+    w1 = 1.0 / (1.0 + math.exp(l2 - l1))
+    np.testing.assert_allclose(w1 * o1 + (1 - w1) * o2, whole, rtol=0, atol=1e-13)
+
+
+def test_float32_twin_agrees():
+    n = 300
+    q, K, V = rnd(9, 0, (64,)), rnd(9, 1, (n, 64)), rnd(9, 2, (n, 64))
+    a, pa = oracle.attend(q, K, V)
+    b, pb = oracle.attend(q, K, V, f32=True)
+    assert b.dtype == np.float32
+    np.testing.assert_allclose(a, b, rtol=0, atol=1e-5)
+    np.testing.assert_allclose(pa, pb, rtol=0, atol=1e-6)
+
+
+# ---------------------------------------------------------------- brute force, library routine
+
+def brute_force(q, K, V, scale):
+    """Pure-Python restatement with Python floats; only for tiny inputs."""
+    n, hd = len(K), len(q)
+    s = [scale * sum(q[d] * K[j][d] for d in range(hd)) for j in range(n)]
+    m = max(s)
+    e = [math.exp(x - m) for x in s]
+    z = sum(e)
+    return [sum(e[j] / z * V[j][d] for j in range(n)) for d in range(hd)]
+
+
+@pytest.mark.parametrize("n,hd", [(1, 4), (3, 4), (6, 8), (11, 8)])
+def test_brute_force_tiny(n, hd):
+    q, K, V = rnd(10, n, (hd,)), rnd(10, 50 + n, (n, hd)), rnd(10, 90 + n, (n, hd))
+    out, _ = oracle.attend(q, K, V, scale=0.5)
+    ref = brute_force(widen(q).tolist(), widen(K).tolist(), widen(V).tolist(), 0.5)
+    np.testing.assert_allclose(out, ref, rtol=0, atol=1e-13)
+
+
+def sdpa64(q, k, v, causal):
+    t = lambda b: torch.from_numpy(widen(b))
+    return torch.nn.functional.scaled_dot_product_attention(t(q), t(k), t(v), is_causal=causal).numpy()
+
+
+def test_prefill_matches_library_causal_attention():
+    B, H, T, hd = 2, 3, 37, 32
+    q, k, v = rnd(11, 0, (B, H, T, hd)), rnd(11, 1, (B, H, T, hd)), rnd(11, 2, (B, H, T, hd))
+    np.testing.assert_allclose(oracle.block_prefill_attn(q, k, v), sdpa64(q, k, v, True), rtol=0, atol=1e-12)
+
+
+def test_prefill_is_not_the_transposed_or_unmasked_variant():
+    # a mistake the library pin must see: no mask, or mask on the wrong side
+    B, H, T, hd = 1, 1, 9, 8
+    q, k, v = rnd(12, 0, (B, H, T, hd)), rnd(12, 1, (B, H, T, hd)), rnd(12, 2, (B, H, T, hd))
+    out = oracle.block_prefill_attn(q, k, v)
+    assert np.abs(out - sdpa64(q, k, v, False)).max() > 1e-3
+    # row 0 sees only block 0
+    np.testing.assert_allclose(out[0, 0, 0], widen(v[0, 0, 0]), rtol=0, atol=0)
+    # last row sees everything: equals the unmasked library result for that row
+    np.testing.assert_allclose(out[0, 0, -1], sdpa64(q, k, v, False)[0, 0, -1], rtol=0, atol=1e-12)
+
+
+def test_prefill_honours_kv_stride():
+    B, H, T, hd, cap = 2, 2, 5, 8, 9
+    q = rnd(13, 0, (B, H, T, hd))
+    k, v = rnd(13, 1, (B, H, cap, hd)), rnd(13, 2, (B, H, cap, hd))
+    a = oracle.block_prefill_attn(q, k, v)
+    b = oracle.block_prefill_attn(q, np.ascontiguousarray(k[:, :, :T]), np.ascontiguousarray(v[:, :, :T]))
+    assert np.array_equal(a, b)
+
+
+# ---------------------------------------------------------------- invariants the paper fixes
+
+def test_cached_decode_equals_full_recompute():
+    """KV caching changes cost, not the function: step-by-step append + decode reproduces the
+    rows of the dense causal prefill."""
+    B, H, T, hd = 3, 2, 21, 16
+    q, k, v = rnd(14, 0, (B, H, T, hd)), rnd(14, 1, (B, H, T, hd)), rnd(14, 2, (B, H, T, hd))
+    full = oracle.block_prefill_attn(q, k, v)
+    c = oracle.Cache(B, H, T, hd)
+    for t in range(T):
+        oracle.kv_append(c, k[:, :, t:t + 1], v[:, :, t:t + 1])
+        assert (c.len == t + 1).all()
+        out = oracle.block_decode_attn(c, np.ascontiguousarray(q[:, :, t]))
+        assert np.array_equal(out, full[:, :, t])
+    assert np.array_equal(c.k, k) and np.array_equal(c.v, v) and c.status[0] == 0
+
+
+def test_block_length_one_is_vanilla_causal_attention():
+    """At L_B = 1 every token is its own block, so block-decoder attention over the block cache
+    is token-level causal attention (the library routine, float64)."""
+    B, H, L, hd = 2, 2, 24, 16
+    q, k, v = rnd(15, 0, (B, H, L, hd)), rnd(15, 1, (B, H, L, hd)), rnd(15, 2, (B, H, L, hd))
+    ref = sdpa64(q, k, v, True)
+    c = oracle.Cache(B, H, L, hd)
+    for t in range(L):
+        oracle.kv_append(c, k[:, :, t:t + 1], v[:, :, t:t + 1])
+        out = oracle.block_decode_attn(c, np.ascontiguousarray(q[:, :, t]))
+        np.testing.assert_allclose(out, ref[:, :, t], rtol=0, atol=1e-12)
+
+
+def test_ragged_lengths_and_rows_past_len_are_ignored():
+    B, H, cap, hd = 4, 2, 12, 8
+    c = oracle.Cache(B, H, cap, hd)
+    c.k[...] = rnd(16, 1, c.k.shape)
+    c.v[...] = rnd(16, 2, c.v.shape)
+    c.len[...] = [1, 5, 12, 7]
+    q = rnd(16, 0, (B, H, hd))
+    out = oracle.block_decode_attn(c, q)
+    for b in range(B):
+        n = c.len[b]
+        ref = sdpa64(q[b][:, None, :], c.k[b, :, :n], c.v[b, :, :n], False)[:, 0]
+        np.testing.assert_allclose(out[b], ref, rtol=0, atol=1e-12)
+    c2 = c.copy()
+    for b in range(B):
+        c2.k[b, :, c.len[b]:] = 0x7FC0  # NaN beyond the length
+        c2.v[b, :, c.len[b]:] = 0x7FC0
+    assert np.array_equal(oracle.block_decode_attn(c2, q), out)
+
+
+def test_spike_row_at_the_length_boundary():
+    """A key far above the rest flips the output to its value: inside the length it must win,
+    one past the length it must be invisible (an off-by-one in the row range fails here)."""
+    B, H, cap, hd, n = 1, 1, 40, 8, 31
+    c = oracle.Cache(B, H, cap, hd)
+    c.k[...] = rnd(17, 1, c.k.shape)
+    c.v[...] = rnd(17, 2, c.v.shape)
+    c.len[...] = n
+    q = bits(np.full((B, H, hd), 3.0))
+    base = oracle.block_decode_attn(c, q)
+    spike_k, spike_v = bits(np.full(hd, 30.0)), bits(np.arange(hd) + 100.0)
+    for row, visible in ((0, True), (n - 1, True), (n, False)):
+        d = c.copy()
+        d.k[0, 0, row], d.v[0, 0, row] = spike_k, spike_v
+        out = oracle.block_decode_attn(d, q)
+        if visible:
+            np.testing.assert_allclose(out[0, 0], widen(spike_v), rtol=0, atol=1e-6)
+        else:
+            assert np.array_equal(out, base)
+
+
+def test_append_overflow_and_empty_cache():
+    c = oracle.Cache(2, 1, 3, 8)
+    c.len[...] = [2, 3]
+    k, v = rnd(18, 1, (2, 1, 1, 8)), rnd(18, 2, (2, 1, 1, 8))
+    oracle.kv_append(c, k, v)
+    assert c.len.tolist() == [3, 3] and c.status[0] == oracle.ST_OVERFLOW
+    assert np.array_equal(c.k[0, 0, 2], k[0, 0, 0]) and not c.k[1].any()
+    e = oracle.Cache(1, 1, 3, 8)
+    out = oracle.block_decode_attn(e, rnd(18, 0, (1, 1, 8)))
+    assert not out.any() and e.status[0] == oracle.ST_EMPTY
+
+
+# ---------------------------------------------------------------- token decoder
+
+def run_token_blocks(L_B, P, n_blocks, seed, B=2, H=2, hd=8, poison_between=False):
+    """Drive the fused token step over n_blocks blocks following the schedule model."""
+    c = oracle.Cache(B, H, P + L_B, hd)
+    outs, lens = [], []
+    for t, (reset, n_app, len_after) in enumerate(oracle.token_step_schedule(L_B, P, n_blocks * L_B)):
+        q, k, v = (rnd(seed, 10 * t + i, (B, H, n_app, hd)) for i in range(3))
+        if reset and poison_between:
+            c.k[...] = rnd(seed + 99, t, c.k.shape)  # whatever the finished block left behind
+            c.v[...] = 0x7FC0
+        outs.append(oracle.token_decode_attn(c, q, k, v, reset_first=bool(reset)))
+        assert (c.len == len_after).all()
+        lens.append(len_after)
+    return outs, lens, c
+
+
+@pytest.mark.parametrize("L_B,P", [(4, 1), (4, 2), (1, 1), (8, 2), (2, 4)])
+def test_token_decoder_never_crosses_a_block_boundary(L_B, P):
+    a, lens, _ = run_token_blocks(L_B, P, 3, seed=20)
+    b, _, _ = run_token_blocks(L_B, P, 3, seed=20, poison_between=True)
+    for x, y in zip(a, b):
+        assert np.array_equal(x, y)
+    assert max(lens) == P + L_B - 1
+
+
+def test_token_step_equals_attention_over_prefix_plus_same_block_tokens():
+    L_B, P, B, H, hd = 4, 2, 2, 2, 8
+    c = oracle.Cache(B, H, P + L_B, hd)
+    ks, vs = [], []
+    for t, (reset, n_app, _) in enumerate(oracle.token_step_schedule(L_B, P, 2 * L_B)):
+        q, k, v = (rnd(21, 10 * t + i, (B, H, n_app, hd)) for i in range(3))
+        if reset:
+            ks, vs = [], []
+        ks.append(k)
+        vs.append(v)
+        out = oracle.token_decode_attn(c, q, k, v, reset_first=bool(reset))
+        Kall, Vall = np.concatenate(ks, 2), np.concatenate(vs, 2)
+        n = Kall.shape[2]
+        for i in range(n_app):  # new row i sees rows 0 .. n - n_app + i
+            m = n - n_app + i + 1
+            ref = sdpa64(q[:, :, i:i + 1], Kall[:, :, :m], Vall[:, :, :m], False)
+            np.testing.assert_allclose(out[:, :, i:i + 1], ref, rtol=0, atol=1e-12)
+
+
+def test_token_attend_only_and_masked_reset():
+    B, H, hd, cap = 3, 1, 8, 5
+    c = oracle.Cache(B, H, cap, hd)
+    for t in range(3):
+        q, k, v = (rnd(22, 10 * t + i, (B, H, 1, hd)) for i in range(3))
+        oracle.token_decode_attn(c, q, k, v)
+    assert c.len.tolist() == [3, 3, 3]
+    q = rnd(22, 77, (B, H, 1, hd))
+    out = oracle.token_decode_attn(c, q, None, None)
+    ref = sdpa64(q, c.k[:, :, :3], c.v[:, :, :3], False)
+    np.testing.assert_allclose(out, ref, rtol=0, atol=1e-12)
+    assert c.len.tolist() == [3, 3, 3]
+    q, k, v = (rnd(22, 90 + i, (B, H, 1, hd)) for i in range(3))
+    out = oracle.token_decode_attn(c, q, k, v, reset_mask=[0, 1, 0])
+    assert c.len.tolist() == [4, 1, 4]
+    np.testing.assert_array_equal(out[1, 0, 0], widen(v[1, 0, 0]))
+    oracle.local_kv_reset(c, mask=[1, 0, 0])
+    assert c.len.tolist() == [0, 1, 4]
+    oracle.local_kv_reset(c)
+    assert c.len.tolist() == [0, 0, 0]
+
+
+def test_token_overflow_is_skipped_and_flagged():
+    B, H, hd, cap = 2, 1, 8, 2
+    c = oracle.Cache(B, H, cap, hd)
+    c.len[...] = [1, 2]
+    q, k, v = (rnd(23, i, (B, H, 1, hd)) for i in range(3))
+    out = oracle.token_decode_attn(c, q, k, v)
+    assert c.len.tolist() == [2, 2] and c.status[0] & oracle.ST_OVERFLOW
+    assert not out[1].any() and not c.k[1].any()
+
+
+# ---------------------------------------------------------------- schedule model + byte model
+
+def golden():
+    vals = {}
+    with open(os.path.join(os.path.dirname(__file__), "golden", "paper_counting_examples.txt")) as f:
+        for line in f:
+            line = line.split("#")[0].strip()
+            if "=" in line:
+                k, v = line.split("=")
+                vals[k.strip()] = int(v)
+    return vals
+
+
+def test_schedule_model():
+    g = golden()
+    s = oracle.token_step_schedule(4, 2, 8)
+    assert [x[2] for x in s] == [2, 3, 4, 5, 2, 3, 4, 5]
+    assert max(x[2] for x in s) == g["local_attn_len_LB4_P2"]
+    assert [x[0] for x in s] == [1, 0, 0, 0, 1, 0, 0, 0]
+    ev = oracle.generation_schedule(4, 1, 128, 2048)
+    assert ev[0] == ("prefill", 32)
+    assert sum(e[0] == "token" for e in ev) == 2048
+    blocks = [e[1] for e in ev if e[0] == "block"]
+    assert blocks == list(range(33, 33 + 512))
+    # L_B = 1: one block step per token, local cache never beyond the prefix
+    ev1 = oracle.generation_schedule(1, 1, 128, 16)
+    assert all(e[3] == 1 and e[1] == 1 for e in ev1 if e[0] == "token")
+
+
+def test_byte_model_matches_the_papers_counting_examples():
+    from workloads import traffic
+    g = golden()
+    per_tok = traffic.kv_bytes_per_token(g["llama7b_layers"], g["llama7b_model_dim"])
+    assert per_tok == g["llama7b_kv_bytes_per_token"]
+    assert per_tok * 2048 * 16 == g["llama7b_kv_bytes_L2048_B16"]
+    # block-decoder KV reads over a generation shrink by L_B^2 (size / L_B, frequency / L_B)
+    def kv_reads(L_B, L=2048, B=1, H=16, hd=64):
+        return sum(B * H * n * 2 * hd * 2 for n in range(1, L // L_B + 1))
+    r = kv_reads(1) / kv_reads(4)
+    assert abs(r / 16 - 1) < 0.01
+    # token-decoder KV reads: L_B^2-ish per block over L/L_B blocks vs L^2  ->  ~ L / L_B
+    L, L_B = 2048, 4
+    vanilla = sum(range(1, L + 1))
+    local = (L // L_B) * sum(range(1, L_B + 1))
+    assert abs((vanilla / local) / (L / L_B) - 1) < 0.25

@@ -1,0 +1,69 @@
+"""Named workload shapes (plain data, no arithmetic of the method).
+
+The shapes follow the paper's model table (12+12 layers, 16 heads, model dim 1024
+with head_dim 64, or 2048 with head_dim 128), its block length L_B = 4 and its
+two serving settings: prefill-heavy (2048 prompt / 128 generated) and
+decode-heavy (128 / 2048), with every prompt padded to the same length.
+"""
+from __future__ import annotations
+
+from dataclasses import dataclass, replace
+
+
+@dataclass(frozen=True)
+class Workload:
+    name: str
+    batch: int
+    heads: int
+    head_dim: int
+    block_len: int          # L_B
+    prefix_len: int         # P
+    n_layers: int
+    max_blocks: int         # block-cache capacity N_max (rows)
+    ctx_blocks: int = 0     # block-cache length after the append (decode configs)
+    prompt_blocks: int = 0  # T (prefill configs)
+    prompt_tokens: int = 0
+    gen_tokens: int = 0
+    seed: int = 1000
+
+    @property
+    def local_cap(self) -> int:
+        return self.prefix_len + self.block_len
+
+
+# config 1: tiny single decode step, every entry point, checked against full recompute
+TINY = Workload("tiny", batch=4, heads=8, head_dim=64, block_len=4, prefix_len=1, n_layers=2,
+                max_blocks=64, ctx_blocks=64, prompt_blocks=64, seed=1001)
+
+# config 2: block-decoder decode step (2048-token context -> 512 block entries), 12 layers
+BLOCK_DECODE = Workload("block_decode", batch=256, heads=16, head_dim=64, block_len=4, prefix_len=1,
+                        n_layers=12, max_blocks=512, ctx_blocks=512, seed=1002)
+
+# config 3: token-decoder local decode, 4096 sequences, local cache 1 prefix + up to L_B tokens
+TOKEN_DECODE = Workload("token_decode", batch=4096, heads=16, head_dim=64, block_len=4, prefix_len=1,
+                        n_layers=12, max_blocks=1, gen_tokens=4096, seed=1003)
+
+# config 4: block-decoder prefill, 2048-token prompt -> 512 blocks, head_dim 128
+BLOCK_PREFILL = Workload("block_prefill", batch=32, heads=16, head_dim=128, block_len=4, prefix_len=1,
+                         n_layers=12, max_blocks=512, prompt_blocks=512, prompt_tokens=2048, seed=1004)
+
+# config 4b: the 8K-prompt case (2048 blocks), where the tensor pipe rather than HBM binds
+BLOCK_PREFILL_8K = Workload("block_prefill_8k", batch=8, heads=16, head_dim=128, block_len=4, prefix_len=1,
+                            n_layers=12, max_blocks=2048, prompt_blocks=2048, prompt_tokens=8192, seed=1014)
+
+
+def sweep(block_len: int) -> Workload:
+    """config 5: decode-heavy generation (128-token prompt, 2048 generated) at one block length."""
+    prompt, gen = 128, 2048
+    return Workload(f"sweep_LB{block_len}", batch=512, heads=16, head_dim=64, block_len=block_len,
+                    prefix_len=1, n_layers=12, max_blocks=(prompt + gen) // block_len,
+                    prompt_blocks=prompt // block_len, prompt_tokens=prompt, gen_tokens=gen,
+                    seed=1005)
+
+
+def scaled(w: Workload, **kw) -> Workload:
+    """A smaller copy of a workload for tests (same structure, fewer sequences/layers)."""
+    return replace(w, **kw)
+
+
+BY_NAME = {w.name: w for w in (TINY, BLOCK_DECODE, TOKEN_DECODE, BLOCK_PREFILL, BLOCK_PREFILL_8K)}

@@ -1,0 +1,43 @@
+"""Algorithmic byte and FLOP counts of the attention path (cost model only).
+
+These are the numbers the roofline fractions are quoted against: the bytes an
+ideal implementation must move once, with bf16 (2-byte) storage.  The formulas
+are checked against the paper's own counting examples (KV bytes per token of a
+7B model; L_B**2 and L/L_B reductions) in the CPU tests.
+"""
+from __future__ import annotations
+
+BF16 = 2
+
+
+def kv_bytes_per_token(n_layers: int, model_dim: int, elem_bytes: int = BF16) -> int:
+    """K and V of one position over all layers."""
+    return n_layers * 2 * model_dim * elem_bytes
+
+
+def block_decode_layer_bytes(B: int, H: int, hd: int, ctx_len: int, with_append: bool = True) -> int:
+    """One layer of one block-decoder decode step: read K,V rows 0..ctx_len-1, q in, out out,
+    and (if fused in the step) the appended row read once and written once."""
+    kv = B * H * ctx_len * 2 * hd * BF16
+    qo = 2 * B * H * hd * BF16
+    app = (2 * 2 * B * H * hd * BF16) if with_append else 0
+    return kv + qo + app
+
+
+def token_decode_layer_bytes(B: int, H: int, hd: int, rows_before: int, n_new: int = 1) -> int:
+    """One layer of one token-decoder step: q, k_new, v_new in; out out; the new rows written
+    to the local cache; rows_before cached rows (K and V) read."""
+    row = hd * BF16
+    fixed = (3 * n_new + n_new + 2 * n_new) * row      # q,k,v reads + out write + K,V row writes
+    return B * H * (fixed + rows_before * 2 * row)
+
+
+def prefill_layer_bytes(B: int, H: int, T: int, hd: int) -> int:
+    """Q, K, V read once and the output written once."""
+    return 4 * B * H * T * hd * BF16
+
+
+def prefill_layer_flops(B: int, H: int, T: int, hd: int) -> int:
+    """Causal attention: T(T+1)/2 (query, key) pairs, each 2*hd flops for the score and 2*hd
+    for the weighted sum."""
+    return B * H * (T * (T + 1) // 2) * 4 * hd
