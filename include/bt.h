@@ -1,0 +1,184 @@
+/*
+ * bt.h - C ABI of the Block Transformer KV-cache attention library (sm_100a).
+ *
+ * The library implements the attention that reads the KV cache in the Block
+ * Transformer's two decoders (paper sections 2.3 and 2.4, appendix E.2):
+ *   - block decoder: causal attention over a block-level KV cache with one row per
+ *     L_B-token block, run once every L_B tokens (decode) or over all prompt blocks
+ *     at once (prefill);
+ *   - token decoder: attention confined to the current block, over a small local
+ *     KV cache seeded by P prefix rows and dropped at every block boundary.
+ *
+ * Conventions
+ *   - Every data pointer is DEVICE memory owned by the caller unless an argument
+ *     is explicitly named *_host.  The library never allocates, frees or keeps
+ *     device memory.
+ *   - bf16 storage, fp32 arithmetic.  Outputs are bf16, rounded to nearest even
+ *     from the fp32 accumulators.  Lengths are int32.
+ *   - q / k_new / v_new / out tensors are contiguous [B][H][n][hd] (n = 1 may be
+ *     thought of as [B][H][hd]).
+ *   - `stream` is a cudaStream_t passed as void*.  All work is enqueued on it and
+ *     the call returns without synchronising.
+ *   - Host-detectable errors (null pointer, bad shape, unsupported head_dim, a
+ *     request larger than the capacity, workspace too small) return a non-zero
+ *     bt_status before anything is launched.  Data-dependent conditions found on
+ *     the device (a sequence whose cache is full, attention over an empty cache)
+ *     never trap: the sequence is skipped or zeros are produced, and a BT_DEV_*
+ *     bit is OR-ed into *dev_status (a device uint32 the caller clears and reads
+ *     when it chooses; may be NULL to ignore).
+ *   - softmax scale: cfg->softmax_scale, or 1/sqrt(head_dim) when it is 0 (the
+ *     paper uses the Pythia / GPT-NeoX architecture and does not restate it).
+ *   - Positions: the library is position-agnostic; rotary or other position
+ *     encodings are applied by the caller before K is cached.
+ */
+#ifndef BT_H_
+#define BT_H_
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef enum {
+    BT_OK = 0,
+    BT_ERR_NULL = 1,        /* a required pointer is NULL                         */
+    BT_ERR_SHAPE = 2,       /* non-positive or inconsistent dimension, bad layer  */
+    BT_ERR_UNSUPPORTED = 3, /* head_dim not in {64,128}, too many heads, ...      */
+    BT_ERR_CAPACITY = 4,    /* n_new larger than the cache capacity               */
+    BT_ERR_WORKSPACE = 5,   /* workspace NULL or smaller than bt_workspace_bytes  */
+    BT_ERR_CUDA = 6         /* a CUDA runtime call or launch failed               */
+} bt_status;
+
+/* bits of the device status word */
+enum { BT_DEV_OK = 0, BT_DEV_OVERFLOW = 1, BT_DEV_EMPTY = 2, BT_DEV_TIMEOUT = 4 };
+
+/* Problem statement in the paper's terms (section 2; model table in appendix D). */
+typedef struct bt_config {
+    int32_t batch;         /* B: sequences decoded together                          */
+    int32_t heads;         /* H: attention heads (plain multi-head: one K,V per head) */
+    int32_t head_dim;      /* hd: 64 or 128                                          */
+    int32_t block_len;     /* L_B: tokens per block, >= 1                            */
+    int32_t prefix_len;    /* P: prefix rows projected from the context embedding    */
+    int32_t max_blocks;    /* N_max: block-cache capacity in rows (= blocks)         */
+    int32_t n_layers;      /* caches and length arrays hold this many layers         */
+    int32_t decode_splits; /* 0: library chooses how many ways bt_block_decode_attn
+                              splits the row range; >0: forced (tests, tuning)       */
+    float softmax_scale;   /* 0 => 1/sqrt(head_dim)                                  */
+} bt_config;
+
+/* Block-level KV cache (section 2.3): one row per block.
+ *   k, v : bf16 [n_layers][B][H][N_max][hd]
+ *   len  : int32 [n_layers][B]   rows valid per (layer, sequence)                   */
+typedef struct bt_block_cache {
+    void* k;
+    void* v;
+    int32_t* len;
+} bt_block_cache;
+
+/* Local KV cache of the token decoder (section 2.4): capacity C = P + L_B rows, K and V
+ * rows interleaved so that one (sequence, head) is one contiguous run.
+ *   kv  : bf16 [n_layers][B][H][C][2][hd]   ([..][c][0][:] = K row c, [..][c][1][:] = V row c)
+ *   len : int32 [n_layers][B]                                                       */
+typedef struct bt_local_cache {
+    void* kv;
+    int32_t* len;
+} bt_local_cache;
+
+/* Library version (major*10000 + minor*100 + patch) and a printable status name. */
+int bt_version(void);
+const char* bt_status_string(bt_status s);
+
+/* Number of ways bt_block_decode_attn will split each (sequence, head) row range for this
+ * config (>= 1), and the workspace it then needs: splits * B * H * (hd + 4) floats when
+ * splits > 1, else 0.  Both return 0 on an invalid config.                              */
+int bt_decode_splits(const bt_config* cfg);
+size_t bt_workspace_bytes(const bt_config* cfg);
+
+/*
+ * Block-decoder KV append (sections 2.1 and 2.3: the K,V of every processed block are cached,
+ * one row per block, written once every L_B tokens; n_new = T writes a whole prefilled prompt).
+ * For each sequence b: rows len[b] .. len[b]+n_new-1 of every head receive k_new / v_new
+ * [B][H][n_new][hd], then len[b] += n_new.  A sequence with len[b] + n_new > N_max is left
+ * untouched and BT_DEV_OVERFLOW is raised.  Returns BT_ERR_CAPACITY if n_new > N_max.
+ */
+bt_status bt_block_kv_append(const bt_config* cfg, bt_block_cache* cache, int layer,
+                             const void* k_new, const void* v_new, int n_new,
+                             uint32_t* dev_status, void* stream);
+
+/*
+ * Block-decoder decode attention (section 2.3; appendix E.2 "decode IO"): for each (b,h),
+ *   out[b,h,:] = sum_j softmax_j(scale * q[b,h,:] . K[b,h,j,:]) * V[b,h,j,:],  j < len[b],
+ * i.e. the query of the newest block attends to every cached block including its own row
+ * len[b]-1.  q, out: [B][H][hd].  len[b] == 0 gives zeros and BT_DEV_EMPTY.
+ * workspace: device scratch of at least bt_workspace_bytes(cfg) bytes (may be NULL when that
+ * is 0); it holds the per-split partial results and needs no initialisation.
+ */
+bt_status bt_block_decode_attn(const bt_config* cfg, const bt_block_cache* cache, int layer,
+                               const void* q, void* out, void* workspace, size_t workspace_bytes,
+                               uint32_t* dev_status, void* stream);
+
+/*
+ * Block boundary of the token decoder (Figure 1; section 2.4): the local K,V of a finished
+ * block are never read again, so the cache is dropped by zeroing its length; no data is
+ * cleared.  seq_mask: NULL resets every sequence, else uint8 [B], non-zero = reset.
+ */
+bt_status bt_local_kv_reset(const bt_config* cfg, bt_local_cache* cache, int layer,
+                            const uint8_t* seq_mask, void* stream);
+
+/*
+ * Append n_new rows to the local cache without attending (section 2.4: prefix rows, or the
+ * partially filled most recent prompt block, the only prompt tokens the token decoder sees).
+ * Same semantics as bt_block_kv_append with capacity C = P + L_B.
+ */
+bt_status bt_local_kv_append(const bt_config* cfg, bt_local_cache* cache, int layer,
+                             const void* k_new, const void* v_new, int n_new,
+                             uint32_t* dev_status, void* stream);
+
+/*
+ * Fused token-decoder step (section 2.4; appendix E.2): in one launch, per sequence b,
+ *   1. reset:  if reset_mask ? reset_mask[b] : reset_first, then len[b] = 0 (block boundary);
+ *   2. append: rows len[b] .. len[b]+n_q-1 receive k_new / v_new [B][H][n_q][hd];
+ *   3. attend: new row i (i < n_q) attends to local rows 0 .. len_old+i, i.e. the prefix rows,
+ *      the earlier tokens of the same block and itself - never anything outside the block;
+ *   4. len[b] += n_q.
+ * n_q = 1 for a token step; n_q = P at a block start appends the P prefix rows, causally
+ * masked among themselves.  k_new == v_new == NULL: nothing is appended, n_q must be 1 and
+ * the query attends to rows 0 .. len[b]-1 (zeros and BT_DEV_EMPTY if there are none).
+ * A sequence without room for n_q rows is skipped: nothing written, zeros out,
+ * BT_DEV_OVERFLOW.  q, out: [B][H][n_q][hd].
+ */
+bt_status bt_token_decode_attn(const bt_config* cfg, bt_local_cache* cache, int layer,
+                               const void* q, const void* k_new, const void* v_new, int n_q,
+                               int reset_first, const uint8_t* reset_mask, void* out,
+                               uint32_t* dev_status, void* stream);
+
+/*
+ * Block-decoder prefill attention (sections 2.1 and 2.3: the prefill stage processes all
+ * prompt positions in parallel; the block decoder does so over T = L / L_B blocks):
+ *   out[b,h,t,:] = sum_{j<=t} softmax_j(scale * q[b,h,t,:] . k[b,h,j,:]) * v[b,h,j,:],  t < T.
+ * q, out: [B][H][T][hd].  k, v: rows hd apart; (b,h) slab s starts s * kv_seq_stride rows
+ * after the base, so kv_seq_stride = T for packed tensors and = N_max when k, v point at a
+ * layer of a block cache that already holds the prompt's rows.  Requires kv_seq_stride >= T.
+ */
+bt_status bt_block_prefill_attn(const bt_config* cfg, const void* q, const void* k, const void* v,
+                                int n_blocks, int64_t kv_seq_stride, void* out, void* stream);
+
+/*
+ * One block-decoder decode step of one layer driven from HOST buffers (the same operations as
+ * bt_block_kv_append followed by bt_block_decode_attn, section 2.3): q_host, k_new_host,
+ * v_new_host [B][H][hd] bf16 are copied to the caller's device staging buffers q_dev, k_dev,
+ * v_dev, the row is appended, attention runs, and out_dev is copied to out_host [B][H][hd].
+ * Host buffers should be pinned; all copies are asynchronous on `stream`.
+ */
+bt_status bt_block_decode_step_host(const bt_config* cfg, bt_block_cache* cache, int layer,
+                                    const void* q_host, const void* k_new_host, const void* v_new_host,
+                                    void* out_host, void* q_dev, void* k_dev, void* v_dev, void* out_dev,
+                                    void* workspace, size_t workspace_bytes, uint32_t* dev_status,
+                                    void* stream);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* BT_H_ */

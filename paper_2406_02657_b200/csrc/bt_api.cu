@@ -1,0 +1,250 @@
+// C-ABI layer: argument validation, layer offsets, dispatch to the kernels.
+// Nothing here touches device memory on the host side or allocates any.
+#include <math.h>
+
+#include "../../include/bt.h"
+#include "bt_kernels.h"
+
+namespace {
+
+constexpr float kLog2e = 1.4426950408889634f;
+
+bool config_ok(const bt_config* c)
+{
+    return c && c->batch > 0 && c->heads > 0 && c->head_dim > 0 && c->block_len > 0 && c->prefix_len > 0 &&
+           c->max_blocks > 0 && c->n_layers > 0 && c->decode_splits >= 0 && c->softmax_scale >= 0.f &&
+           isfinite(c->softmax_scale);
+}
+
+bt_status check_config(const bt_config* c, int layer)
+{
+    if (!c) return BT_ERR_NULL;
+    if (!config_ok(c)) return BT_ERR_SHAPE;
+    if (layer < 0 || layer >= c->n_layers) return BT_ERR_SHAPE;
+    if (c->head_dim != 64 && c->head_dim != 128) return BT_ERR_UNSUPPORTED;
+    if (c->heads * (c->head_dim / 8) > 256) return BT_ERR_UNSUPPORTED;  // one CTA must cover a sequence
+    if (c->decode_splits > 64) return BT_ERR_UNSUPPORTED;
+    return BT_OK;
+}
+
+float scale_log2(const bt_config* c)
+{
+    const float s = c->softmax_scale > 0.f ? c->softmax_scale : 1.0f / sqrtf((float)c->head_dim);
+    return s * kLog2e;
+}
+
+int choose_splits(const bt_config* c)
+{
+    if (c->decode_splits > 0) return c->decode_splits;
+    // enough CTAs for a few per SM; never fewer than 16 rows per split
+    const long long bh = (long long)c->batch * c->heads;
+    const long long target = 148 * 4;
+    long long s = (target + bh - 1) / bh;
+    long long by_rows = c->max_blocks / 16;
+    if (by_rows < 1) by_rows = 1;
+    if (s > by_rows) s = by_rows;
+    if (s > 32) s = 32;
+    if (s < 1) s = 1;
+    return (int)s;
+}
+
+inline size_t block_layer_elems(const bt_config* c) { return (size_t)c->batch * c->heads * c->max_blocks * c->head_dim; }
+inline int local_cap(const bt_config* c) { return c->prefix_len + c->block_len; }
+inline size_t local_layer_elems(const bt_config* c) { return (size_t)c->batch * c->heads * local_cap(c) * 2 * c->head_dim; }
+
+bt::CacheView block_view(const bt_config* c, const bt_block_cache* cache, int layer)
+{
+    bt::CacheView v;
+    v.k = (char*)cache->k + block_layer_elems(c) * layer * 2;
+    v.v = (char*)cache->v + block_layer_elems(c) * layer * 2;
+    v.len = cache->len + (size_t)layer * c->batch;
+    v.slab_stride = (int64_t)c->max_blocks * c->head_dim;
+    v.row_stride = c->head_dim;
+    v.cap = c->max_blocks;
+    return v;
+}
+
+bt::CacheView local_view(const bt_config* c, const bt_local_cache* cache, int layer)
+{
+    bt::CacheView v;
+    char* base = (char*)cache->kv + local_layer_elems(c) * layer * 2;
+    v.k = base;
+    v.v = base + (size_t)c->head_dim * 2;
+    v.len = cache->len + (size_t)layer * c->batch;
+    v.slab_stride = (int64_t)local_cap(c) * 2 * c->head_dim;
+    v.row_stride = 2 * c->head_dim;
+    v.cap = local_cap(c);
+    return v;
+}
+
+inline bt_status cuda_status(cudaError_t e) { return e == cudaSuccess ? BT_OK : BT_ERR_CUDA; }
+
+}  // namespace
+
+extern "C" {
+
+int bt_version(void) { return 100; }
+
+const char* bt_status_string(bt_status s)
+{
+    switch (s) {
+        case BT_OK: return "BT_OK";
+        case BT_ERR_NULL: return "BT_ERR_NULL";
+        case BT_ERR_SHAPE: return "BT_ERR_SHAPE";
+        case BT_ERR_UNSUPPORTED: return "BT_ERR_UNSUPPORTED";
+        case BT_ERR_CAPACITY: return "BT_ERR_CAPACITY";
+        case BT_ERR_WORKSPACE: return "BT_ERR_WORKSPACE";
+        case BT_ERR_CUDA: return "BT_ERR_CUDA";
+    }
+    return "BT_ERR_?";
+}
+
+int bt_decode_splits(const bt_config* cfg)
+{
+    if (check_config(cfg, 0) != BT_OK) return 0;
+    return choose_splits(cfg);
+}
+
+size_t bt_workspace_bytes(const bt_config* cfg)
+{
+    if (check_config(cfg, 0) != BT_OK) return 0;
+    const int s = choose_splits(cfg);
+    if (s <= 1) return 0;
+    return (size_t)s * cfg->batch * cfg->heads * (cfg->head_dim + 4) * sizeof(float);
+}
+
+bt_status bt_block_kv_append(const bt_config* cfg, bt_block_cache* cache, int layer, const void* k_new,
+                             const void* v_new, int n_new, uint32_t* dev_status, void* stream)
+{
+    bt_status st = check_config(cfg, layer);
+    if (st != BT_OK) return st;
+    if (!cache || !cache->k || !cache->v || !cache->len || !k_new || !v_new) return BT_ERR_NULL;
+    if (n_new <= 0) return BT_ERR_SHAPE;
+    if (n_new > cfg->max_blocks) return BT_ERR_CAPACITY;
+    return cuda_status(bt::launch_kv_append(block_view(cfg, cache, layer), cfg->batch, cfg->heads, cfg->head_dim,
+                                            k_new, v_new, n_new, dev_status, (cudaStream_t)stream));
+}
+
+bt_status bt_block_decode_attn(const bt_config* cfg, const bt_block_cache* cache, int layer, const void* q,
+                               void* out, void* workspace, size_t workspace_bytes, uint32_t* dev_status,
+                               void* stream)
+{
+    bt_status st = check_config(cfg, layer);
+    if (st != BT_OK) return st;
+    if (!cache || !cache->k || !cache->v || !cache->len || !q || !out) return BT_ERR_NULL;
+    const size_t need = bt_workspace_bytes(cfg);
+    if (need && (!workspace || workspace_bytes < need)) return BT_ERR_WORKSPACE;
+    bt::CacheView v = block_view(cfg, cache, layer);
+    bt::DecodeArgs a;
+    a.q = q;
+    a.k = v.k;
+    a.v = v.v;
+    a.len = v.len;
+    a.out = out;
+    a.ws = (float*)workspace;
+    a.dev_status = dev_status;
+    a.B = cfg->batch;
+    a.H = cfg->heads;
+    a.hd = cfg->head_dim;
+    a.n_max = cfg->max_blocks;
+    a.splits = choose_splits(cfg);
+    a.scale_log2 = scale_log2(cfg);
+    return cuda_status(bt::launch_block_decode(a, (cudaStream_t)stream));
+}
+
+bt_status bt_local_kv_reset(const bt_config* cfg, bt_local_cache* cache, int layer, const uint8_t* seq_mask,
+                            void* stream)
+{
+    bt_status st = check_config(cfg, layer);
+    if (st != BT_OK) return st;
+    if (!cache || !cache->len) return BT_ERR_NULL;
+    return cuda_status(bt::launch_len_reset(cache->len + (size_t)layer * cfg->batch, cfg->batch, seq_mask,
+                                            (cudaStream_t)stream));
+}
+
+bt_status bt_local_kv_append(const bt_config* cfg, bt_local_cache* cache, int layer, const void* k_new,
+                             const void* v_new, int n_new, uint32_t* dev_status, void* stream)
+{
+    bt_status st = check_config(cfg, layer);
+    if (st != BT_OK) return st;
+    if (!cache || !cache->kv || !cache->len || !k_new || !v_new) return BT_ERR_NULL;
+    if (n_new <= 0) return BT_ERR_SHAPE;
+    if (n_new > local_cap(cfg)) return BT_ERR_CAPACITY;
+    return cuda_status(bt::launch_kv_append(local_view(cfg, cache, layer), cfg->batch, cfg->heads, cfg->head_dim,
+                                            k_new, v_new, n_new, dev_status, (cudaStream_t)stream));
+}
+
+bt_status bt_token_decode_attn(const bt_config* cfg, bt_local_cache* cache, int layer, const void* q,
+                               const void* k_new, const void* v_new, int n_q, int reset_first,
+                               const uint8_t* reset_mask, void* out, uint32_t* dev_status, void* stream)
+{
+    bt_status st = check_config(cfg, layer);
+    if (st != BT_OK) return st;
+    if (!cache || !cache->kv || !cache->len || !q || !out) return BT_ERR_NULL;
+    if ((k_new == nullptr) != (v_new == nullptr)) return BT_ERR_NULL;
+    if (n_q <= 0) return BT_ERR_SHAPE;
+    if (!k_new && n_q != 1) return BT_ERR_SHAPE;
+    if (n_q > local_cap(cfg)) return BT_ERR_CAPACITY;
+    bt::TokenArgs a;
+    a.kv = (char*)cache->kv + local_layer_elems(cfg) * layer * 2;
+    a.len = cache->len + (size_t)layer * cfg->batch;
+    a.q = q;
+    a.k_new = k_new;
+    a.v_new = v_new;
+    a.out = out;
+    a.reset_mask = reset_mask;
+    a.dev_status = dev_status;
+    a.B = cfg->batch;
+    a.H = cfg->heads;
+    a.hd = cfg->head_dim;
+    a.cap = local_cap(cfg);
+    a.n_q = n_q;
+    a.reset_first = reset_first ? 1 : 0;
+    a.scale_log2 = scale_log2(cfg);
+    return cuda_status(bt::launch_token_decode(a, (cudaStream_t)stream));
+}
+
+bt_status bt_block_prefill_attn(const bt_config* cfg, const void* q, const void* k, const void* v, int n_blocks,
+                                int64_t kv_seq_stride, void* out, void* stream)
+{
+    bt_status st = check_config(cfg, 0);
+    if (st != BT_OK) return st;
+    if (!q || !k || !v || !out) return BT_ERR_NULL;
+    if (n_blocks <= 0 || kv_seq_stride < n_blocks) return BT_ERR_SHAPE;
+    bt::PrefillArgs a;
+    a.q = q;
+    a.k = k;
+    a.v = v;
+    a.out = out;
+    a.B = cfg->batch;
+    a.H = cfg->heads;
+    a.hd = cfg->head_dim;
+    a.T = n_blocks;
+    a.kv_seq_stride = kv_seq_stride;
+    a.scale_log2 = scale_log2(cfg);
+    return cuda_status(bt::launch_block_prefill_simple(a, (cudaStream_t)stream));
+}
+
+bt_status bt_block_decode_step_host(const bt_config* cfg, bt_block_cache* cache, int layer, const void* q_host,
+                                    const void* k_new_host, const void* v_new_host, void* out_host, void* q_dev,
+                                    void* k_dev, void* v_dev, void* out_dev, void* workspace,
+                                    size_t workspace_bytes, uint32_t* dev_status, void* stream)
+{
+    bt_status st = check_config(cfg, layer);
+    if (st != BT_OK) return st;
+    if (!q_host || !k_new_host || !v_new_host || !out_host || !q_dev || !k_dev || !v_dev || !out_dev)
+        return BT_ERR_NULL;
+    const size_t bytes = (size_t)cfg->batch * cfg->heads * cfg->head_dim * 2;
+    cudaStream_t s = (cudaStream_t)stream;
+    if (cudaMemcpyAsync(k_dev, k_new_host, bytes, cudaMemcpyHostToDevice, s) != cudaSuccess) return BT_ERR_CUDA;
+    if (cudaMemcpyAsync(v_dev, v_new_host, bytes, cudaMemcpyHostToDevice, s) != cudaSuccess) return BT_ERR_CUDA;
+    if (cudaMemcpyAsync(q_dev, q_host, bytes, cudaMemcpyHostToDevice, s) != cudaSuccess) return BT_ERR_CUDA;
+    st = bt_block_kv_append(cfg, cache, layer, k_dev, v_dev, 1, dev_status, stream);
+    if (st != BT_OK) return st;
+    st = bt_block_decode_attn(cfg, cache, layer, q_dev, out_dev, workspace, workspace_bytes, dev_status, stream);
+    if (st != BT_OK) return st;
+    if (cudaMemcpyAsync(out_host, out_dev, bytes, cudaMemcpyDeviceToHost, s) != cudaSuccess) return BT_ERR_CUDA;
+    return BT_OK;
+}
+
+}  // extern "C"

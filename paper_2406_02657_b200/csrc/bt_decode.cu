@@ -1,0 +1,231 @@
+// Block-decoder decode attention (paper section 2.3; appendix E.2): one query per
+// (sequence, head) over the cached block rows, memory-bound.  Each CTA streams a contiguous
+// range of K and V rows with 128-bit read-once loads, keeps an online softmax per lane and
+// merges lanes, warps and (when the row range is split across CTAs) splits with the
+// log-sum-exp rule.
+#include "bt_common.cuh"
+#include "bt_kernels.h"
+
+namespace bt {
+
+constexpr int kDecodeWarps = 4;
+constexpr int kDecodeThreads = kDecodeWarps * 32;
+constexpr int kUnroll = 8;  // independent K (and V) loads in flight per lane
+// floats per split partial in the workspace: hd outputs + log2-sum-exp, padded so that every
+// partial starts on a 16-byte boundary (the outputs are stored as float4)
+template <int HD>
+constexpr int kPartStride = HD + 4;
+
+// Attention of one query over rows [r0, r1) of one (b,h) slab, by one CTA of kDecodeWarps
+// warps.  On return, threads 0..LPR-1 of warp 0 hold the merged state for their 8 dims
+// (st.acc un-normalised, st.m, st.l identical on those lanes).
+template <int HD>
+__device__ __forceinline__ void attend_range(const bf16* __restrict__ qrow, const bf16* __restrict__ Kb,
+                                             const bf16* __restrict__ Vb, int r0, int r1, float scale_log2,
+                                             SoftmaxState& st, float* smem /* kDecodeWarps*(HD+2) floats */)
+{
+    constexpr int LPR = RowGeo<HD>::LPR, RPW = RowGeo<HD>::RPW;
+    constexpr int TILE = kUnroll * RPW;  // rows per warp iteration
+    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+    const int sub = lane % LPR, rg = lane / LPR;
+
+    float qf[8];
+    {
+        uint4 qr = ld_plain(qrow + sub * 8);
+        unpack8(qr, qf);
+#pragma unroll
+        for (int i = 0; i < 8; ++i) qf[i] *= scale_log2;
+    }
+    st.init();
+
+    for (int base = r0 + warp * TILE; base < r1; base += kDecodeWarps * TILE) {
+        uint4 kr[kUnroll], vr[kUnroll];
+#pragma unroll
+        for (int u = 0; u < kUnroll; ++u) {
+            int row = base + u * RPW + rg;
+            kr[u] = (row < r1) ? ld_stream(Kb + (size_t)row * HD + sub * 8) : make_uint4(0, 0, 0, 0);
+        }
+#pragma unroll
+        for (int u = 0; u < kUnroll; ++u) {
+            int row = base + u * RPW + rg;
+            vr[u] = (row < r1) ? ld_stream(Vb + (size_t)row * HD + sub * 8) : make_uint4(0, 0, 0, 0);
+        }
+        float s[kUnroll];
+        float mt = kNegInf;
+#pragma unroll
+        for (int u = 0; u < kUnroll; ++u) {
+            float d = row_sum<LPR>(dot8(qf, kr[u]));
+            int row = base + u * RPW + rg;
+            s[u] = (row < r1) ? d : kNegInf;
+            mt = fmaxf(mt, s[u]);
+        }
+        if (mt != kNegInf) {  // uniform within the LPR lanes of a row group
+            float mn = fmaxf(st.m, mt);
+            float c = ex2(st.m - mn);
+            st.l *= c;
+#pragma unroll
+            for (int i = 0; i < 8; ++i) st.acc[i] *= c;
+#pragma unroll
+            for (int u = 0; u < kUnroll; ++u) {
+                float p = ex2(s[u] - mn);
+                st.l += p;
+                fma8(st.acc, p, vr[u]);
+            }
+            st.m = mn;
+        }
+    }
+
+    // merge the RPW row groups of the warp
+#pragma unroll
+    for (int off = LPR; off < 32; off <<= 1) {
+        float m2 = __shfl_xor_sync(0xffffffffu, st.m, off);
+        float l2 = __shfl_xor_sync(0xffffffffu, st.l, off);
+        float a2[8];
+#pragma unroll
+        for (int i = 0; i < 8; ++i) a2[i] = __shfl_xor_sync(0xffffffffu, st.acc[i], off);
+        st.merge(m2, l2, a2);
+    }
+    // merge the warps through shared memory
+    if (rg == 0) {
+        float* w = smem + warp * (HD + 2);
+#pragma unroll
+        for (int i = 0; i < 8; ++i) w[sub * 8 + i] = st.acc[i];
+        if (sub == 0) {
+            w[HD] = st.m;
+            w[HD + 1] = st.l;
+        }
+    }
+    __syncthreads();
+    if (warp == 0 && rg == 0) {
+#pragma unroll
+        for (int w2 = 1; w2 < kDecodeWarps; ++w2) {
+            const float* w = smem + w2 * (HD + 2);
+            float a2[8];
+#pragma unroll
+            for (int i = 0; i < 8; ++i) a2[i] = w[sub * 8 + i];
+            st.merge(w[HD], w[HD + 1], a2);
+        }
+    }
+}
+
+// grid: B*H*splits CTAs.  splits == 1 writes bf16 output directly; otherwise each CTA writes
+// its normalised partial (hd floats) and its log2-sum-exp to the workspace.
+template <int HD>
+__global__ void __launch_bounds__(kDecodeThreads) block_decode_kernel(DecodeArgs a)
+{
+    constexpr int LPR = RowGeo<HD>::LPR;
+    __shared__ float smem[kDecodeWarps * (HD + 2)];
+    const int bh = blockIdx.x / a.splits, sp = blockIdx.x - bh * a.splits;
+    const int b = bh / a.H;
+    int n = a.len[b];
+    n = n < 0 ? 0 : (n > a.n_max ? a.n_max : n);
+    const int per = (n + a.splits - 1) / a.splits;
+    const int r0 = min(n, sp * per), r1 = min(n, r0 + per);
+
+    const bf16* Kb = reinterpret_cast<const bf16*>(a.k) + (size_t)bh * a.n_max * HD;
+    const bf16* Vb = reinterpret_cast<const bf16*>(a.v) + (size_t)bh * a.n_max * HD;
+    SoftmaxState st;
+    attend_range<HD>(reinterpret_cast<const bf16*>(a.q) + (size_t)bh * HD, Kb, Vb, r0, r1, a.scale_log2, st, smem);
+
+    if (threadIdx.x < LPR) {
+        const int sub = threadIdx.x;
+        float o[8];
+        float inv = st.l > 0.f ? 1.f / st.l : 0.f;
+#pragma unroll
+        for (int i = 0; i < 8; ++i) o[i] = st.acc[i] * inv;
+        if (a.splits == 1) {
+            *reinterpret_cast<uint4*>(reinterpret_cast<bf16*>(a.out) + (size_t)bh * HD + sub * 8) = pack8(o);
+        } else {
+            float* w = a.ws + ((size_t)bh * a.splits + sp) * kPartStride<HD>;
+            *reinterpret_cast<float4*>(w + sub * 8) = make_float4(o[0], o[1], o[2], o[3]);
+            *reinterpret_cast<float4*>(w + sub * 8 + 4) = make_float4(o[4], o[5], o[6], o[7]);
+            if (sub == 0) w[HD] = st.l > 0.f ? st.m + log2f(st.l) : kNegInf;
+        }
+        if (sub == 0 && sp == 0 && n == 0 && (bh % a.H) == 0) raise_status(a.dev_status, BT_DEV_EMPTY);
+    }
+}
+
+// Combine the per-split partials: out = sum_s w_s o_s with w_s = 2^(lse_s - max) / sum.
+// One lane group of LPR threads per (b,h).
+template <int HD>
+__global__ void __launch_bounds__(128) decode_merge_kernel(DecodeArgs a)
+{
+    constexpr int LPR = RowGeo<HD>::LPR;
+    const int g = (blockIdx.x * blockDim.x + threadIdx.x) / LPR, sub = threadIdx.x % LPR;
+    if (g >= a.B * a.H) return;
+    const float* w = a.ws + (size_t)g * a.splits * kPartStride<HD>;
+    float mx = kNegInf;
+    for (int s = 0; s < a.splits; ++s) mx = fmaxf(mx, w[s * kPartStride<HD> + HD]);
+    float o[8] = {0, 0, 0, 0, 0, 0, 0, 0};
+    float tot = 0.f;
+    if (mx != kNegInf) {
+        for (int s = 0; s < a.splits; ++s) {
+            const float* ws = w + s * kPartStride<HD>;
+            float c = ex2(ws[HD] - mx);
+            tot += c;
+            float4 x = *reinterpret_cast<const float4*>(ws + sub * 8);
+            float4 y = *reinterpret_cast<const float4*>(ws + sub * 8 + 4);
+            o[0] = fmaf(c, x.x, o[0]); o[1] = fmaf(c, x.y, o[1]); o[2] = fmaf(c, x.z, o[2]); o[3] = fmaf(c, x.w, o[3]);
+            o[4] = fmaf(c, y.x, o[4]); o[5] = fmaf(c, y.y, o[5]); o[6] = fmaf(c, y.z, o[6]); o[7] = fmaf(c, y.w, o[7]);
+        }
+        float inv = 1.f / tot;
+#pragma unroll
+        for (int i = 0; i < 8; ++i) o[i] *= inv;
+    }
+    *reinterpret_cast<uint4*>(reinterpret_cast<bf16*>(a.out) + (size_t)g * HD + sub * 8) = pack8(o);
+}
+
+template <int HD>
+static cudaError_t launch_decode_t(const DecodeArgs& a, cudaStream_t stream)
+{
+    const int bh = a.B * a.H;
+    block_decode_kernel<HD><<<bh * a.splits, kDecodeThreads, 0, stream>>>(a);
+    cudaError_t e = cudaGetLastError();
+    if (e != cudaSuccess || a.splits == 1) return e;
+    constexpr int LPR = RowGeo<HD>::LPR;
+    const int groups_per_cta = 128 / LPR;
+    decode_merge_kernel<HD><<<(bh + groups_per_cta - 1) / groups_per_cta, 128, 0, stream>>>(a);
+    return cudaGetLastError();
+}
+
+cudaError_t launch_block_decode(const DecodeArgs& a, cudaStream_t stream)
+{
+    return a.hd == 64 ? launch_decode_t<64>(a, stream) : launch_decode_t<128>(a, stream);
+}
+
+// ---------------------------------------------------------------------------------------
+// Plain prefill: query block t of (b,h) is a decode over rows 0..t (paper section 2.3: the
+// block decoder is causal over blocks).  One CTA per (b,h,t).  Correct for any T; the
+// tensor-core kernel replaces it for the shapes it supports.
+template <int HD>
+__global__ void __launch_bounds__(kDecodeThreads) block_prefill_simple_kernel(PrefillArgs a)
+{
+    constexpr int LPR = RowGeo<HD>::LPR;
+    __shared__ float smem[kDecodeWarps * (HD + 2)];
+    const int bh = blockIdx.x / a.T, t = blockIdx.x - bh * a.T;
+    const bf16* Kb = reinterpret_cast<const bf16*>(a.k) + (size_t)bh * a.kv_seq_stride * HD;
+    const bf16* Vb = reinterpret_cast<const bf16*>(a.v) + (size_t)bh * a.kv_seq_stride * HD;
+    const size_t qoff = ((size_t)bh * a.T + t) * HD;
+    SoftmaxState st;
+    attend_range<HD>(reinterpret_cast<const bf16*>(a.q) + qoff, Kb, Vb, 0, t + 1, a.scale_log2, st, smem);
+    if (threadIdx.x < LPR) {
+        float o[8];
+        float inv = 1.f / st.l;
+#pragma unroll
+        for (int i = 0; i < 8; ++i) o[i] = st.acc[i] * inv;
+        *reinterpret_cast<uint4*>(reinterpret_cast<bf16*>(a.out) + qoff + threadIdx.x * 8) = pack8(o);
+    }
+}
+
+cudaError_t launch_block_prefill_simple(const PrefillArgs& a, cudaStream_t stream)
+{
+    const long long ctas = (long long)a.B * a.H * a.T;
+    if (ctas > 0x7fffffffLL) return cudaErrorInvalidConfiguration;
+    if (a.hd == 64)
+        block_prefill_simple_kernel<64><<<(unsigned)ctas, kDecodeThreads, 0, stream>>>(a);
+    else
+        block_prefill_simple_kernel<128><<<(unsigned)ctas, kDecodeThreads, 0, stream>>>(a);
+    return cudaGetLastError();
+}
+
+}  // namespace bt

@@ -1,0 +1,64 @@
+// Internal launch interface between the C-ABI layer (bt_api.cu) and the kernels.
+// Every launcher enqueues on `stream` and returns the launch's cudaError_t.
+#pragma once
+
+#include <cuda_runtime.h>
+#include <stdint.h>
+
+namespace bt {
+
+// Rows of a cache as the copy kernels see them: K row r of slab s at
+// k + s*slab_stride + r*row_stride (elements), V likewise from v.
+struct CacheView {
+    void* k;
+    void* v;
+    int32_t* len;        // [B] for the layer
+    int64_t slab_stride; // elements between consecutive (b,h) slabs
+    int64_t row_stride;  // elements between consecutive rows
+    int32_t cap;         // rows
+};
+
+cudaError_t launch_kv_append(const CacheView& c, int B, int H, int hd, const void* k_new, const void* v_new,
+                             int n_new, uint32_t* dev_status, cudaStream_t stream);
+cudaError_t launch_len_reset(int32_t* len, int B, const uint8_t* mask, cudaStream_t stream);
+
+struct DecodeArgs {
+    const void* q;       // [B][H][hd]
+    const void* k;       // layer base, [B][H][N_max][hd]
+    const void* v;
+    const int32_t* len;  // [B]
+    void* out;           // [B][H][hd]
+    float* ws;           // [B*H][splits][hd+4] when splits > 1
+    uint32_t* dev_status;
+    int B, H, hd, n_max, splits;
+    float scale_log2;    // softmax scale * log2(e)
+};
+cudaError_t launch_block_decode(const DecodeArgs& a, cudaStream_t stream);
+
+struct TokenArgs {
+    void* kv;            // layer base, [B][H][C][2][hd]
+    int32_t* len;        // [B]
+    const void* q;
+    const void* k_new;   // may be NULL (attend only)
+    const void* v_new;
+    void* out;
+    const uint8_t* reset_mask;
+    uint32_t* dev_status;
+    int B, H, hd, cap, n_q, reset_first;
+    float scale_log2;
+};
+cudaError_t launch_token_decode(const TokenArgs& a, cudaStream_t stream);
+
+struct PrefillArgs {
+    const void* q;
+    const void* k;
+    const void* v;
+    void* out;
+    int B, H, hd, T;
+    int64_t kv_seq_stride;  // rows
+    float scale_log2;
+};
+// Plain CUDA-core kernel: any T, used for shapes the tensor-core kernel does not take.
+cudaError_t launch_block_prefill_simple(const PrefillArgs& a, cudaStream_t stream);
+
+}  // namespace bt

@@ -1,0 +1,99 @@
+"""The C-ABI library loads, exports what include/bt.h declares, and rejects bad arguments
+before launching anything (no GPU needed: every call here returns before a launch)."""
+import ctypes
+import os
+import re
+
+import pytest
+
+ROOT = os.path.dirname(os.path.dirname(os.path.abspath(__file__)))
+
+
+def declared_symbols():
+    text = open(os.path.join(ROOT, "include", "bt.h")).read()
+    text = re.sub(r"/\*.*?\*/", "", text, flags=re.S)
+    return sorted(set(re.findall(r"\b(bt_[a-z0-9_]+)\s*\(", text)))
+
+
+@pytest.fixture(scope="module")
+def bt():
+    import paper_2406_02657_b200 as bt
+    return bt
+
+
+def test_library_exports_every_declared_symbol(bt):
+    names = declared_symbols()
+    assert len(names) >= 11
+    for n in names:
+        assert hasattr(bt.lib(), n), f"{n} declared in bt.h but not exported"
+        assert hasattr(bt, n) or n in ("bt_status_string",), f"{n} has no python binding"
+
+
+def test_version_and_status_strings(bt):
+    assert bt.bt_version() >= 100
+    assert bt.status_string(0) == "BT_OK" and bt.status_string(4) == "BT_ERR_CAPACITY"
+
+
+def test_split_choice_and_workspace(bt):
+    big = bt.make_config(256, 16, 64, 4, 1, 512, 12)
+    assert bt.bt_decode_splits(big) == 1 and bt.bt_workspace_bytes(big) == 0
+    tiny = bt.make_config(4, 8, 64, 4, 1, 64, 2)
+    s = bt.bt_decode_splits(tiny)
+    assert s > 1 and bt.bt_workspace_bytes(tiny) == s * 4 * 8 * 68 * 4
+    forced = bt.make_config(4, 8, 64, 4, 1, 64, 2, decode_splits=7)
+    assert bt.bt_decode_splits(forced) == 7
+    bad = bt.make_config(4, 8, 48, 4, 1, 64, 2)
+    assert bt.bt_decode_splits(bad) == 0 and bt.bt_workspace_bytes(bad) == 0
+
+
+def test_host_detectable_errors_return_before_launch(bt):
+    L = bt.lib()
+    fake = ctypes.c_void_p(0x1000)  # never dereferenced: each call below fails validation first
+    cfg = bt.make_config(4, 8, 64, 4, 1, 64, 2)
+    bc = bt.binding.bt_block_cache(0x1000, 0x1000, 0x1000)
+    lc = bt.binding.bt_local_cache(0x1000, 0x1000)
+    ref = ctypes.byref
+    # null config / bad shapes
+    assert L.bt_block_kv_append(None, ref(bc), 0, fake, fake, 1, None, None) == bt.BT_ERR_NULL
+    assert L.bt_block_kv_append(ref(cfg), ref(bc), 2, fake, fake, 1, None, None) == bt.BT_ERR_SHAPE
+    assert L.bt_block_kv_append(ref(cfg), ref(bc), -1, fake, fake, 1, None, None) == bt.BT_ERR_SHAPE
+    assert L.bt_block_kv_append(ref(cfg), ref(bc), 0, None, fake, 1, None, None) == bt.BT_ERR_NULL
+    assert L.bt_block_kv_append(ref(cfg), ref(bc), 0, fake, fake, 0, None, None) == bt.BT_ERR_SHAPE
+    assert L.bt_block_kv_append(ref(cfg), ref(bc), 0, fake, fake, 65, None, None) == bt.BT_ERR_CAPACITY
+    nullc = bt.binding.bt_block_cache(0, 0x1000, 0x1000)
+    assert L.bt_block_kv_append(ref(cfg), ref(nullc), 0, fake, fake, 1, None, None) == bt.BT_ERR_NULL
+    # unsupported head_dim / too many heads
+    bad = bt.make_config(4, 8, 96, 4, 1, 64, 2)
+    assert L.bt_block_decode_attn(ref(bad), ref(bc), 0, fake, fake, None, 0, None, None) == bt.BT_ERR_UNSUPPORTED
+    many = bt.make_config(4, 64, 64, 4, 1, 64, 2)
+    assert L.bt_block_decode_attn(ref(many), ref(bc), 0, fake, fake, None, 0, None, None) == bt.BT_ERR_UNSUPPORTED
+    neg = bt.make_config(0, 8, 64, 4, 1, 64, 2)
+    assert L.bt_block_decode_attn(ref(neg), ref(bc), 0, fake, fake, None, 0, None, None) == bt.BT_ERR_SHAPE
+    # workspace too small when the row range is split
+    assert L.bt_block_decode_attn(ref(cfg), ref(bc), 0, fake, fake, None, 0, None, None) == bt.BT_ERR_WORKSPACE
+    assert L.bt_block_decode_attn(ref(cfg), ref(bc), 0, fake, fake, fake, 16, None, None) == bt.BT_ERR_WORKSPACE
+    assert L.bt_block_decode_attn(ref(cfg), ref(bc), 0, None, fake, fake, 1 << 20, None, None) == bt.BT_ERR_NULL
+    # local cache
+    assert L.bt_local_kv_reset(ref(cfg), None, 0, None, None) == bt.BT_ERR_NULL
+    assert L.bt_local_kv_append(ref(cfg), ref(lc), 0, fake, fake, 6, None, None) == bt.BT_ERR_CAPACITY
+    assert L.bt_token_decode_attn(ref(cfg), ref(lc), 0, fake, fake, None, 1, 0, None, fake, None, None) == bt.BT_ERR_NULL
+    assert L.bt_token_decode_attn(ref(cfg), ref(lc), 0, fake, None, None, 2, 0, None, fake, None, None) == bt.BT_ERR_SHAPE
+    assert L.bt_token_decode_attn(ref(cfg), ref(lc), 0, fake, fake, fake, 6, 0, None, fake, None, None) == bt.BT_ERR_CAPACITY
+    assert L.bt_token_decode_attn(ref(cfg), ref(lc), 0, fake, fake, fake, 0, 0, None, fake, None, None) == bt.BT_ERR_SHAPE
+    assert L.bt_token_decode_attn(ref(cfg), ref(lc), 0, fake, fake, fake, 1, 0, None, None, None, None) == bt.BT_ERR_NULL
+    # prefill
+    assert L.bt_block_prefill_attn(ref(cfg), fake, fake, fake, 0, 8, fake, None) == bt.BT_ERR_SHAPE
+    assert L.bt_block_prefill_attn(ref(cfg), fake, fake, fake, 16, 8, fake, None) == bt.BT_ERR_SHAPE
+    assert L.bt_block_prefill_attn(ref(cfg), fake, None, fake, 8, 8, fake, None) == bt.BT_ERR_NULL
+    # host-driven step
+    assert L.bt_block_decode_step_host(ref(cfg), ref(bc), 0, None, fake, fake, fake, fake, fake, fake, fake,
+                                       None, 0, None, None) == bt.BT_ERR_NULL
+
+
+def test_oracle_is_not_imported_by_the_product():
+    pkg = os.path.join(ROOT, "paper_2406_02657_b200")
+    for dirpath, _, files in os.walk(pkg):
+        for f in files:
+            if f.endswith((".py", ".cu", ".cuh", ".h")):
+                src = open(os.path.join(dirpath, f)).read()
+                assert "oracle" not in src, f"{f} mentions the oracle"

@@ -1,0 +1,38 @@
+"""Helpers shared by the GPU parity tests (marshalling between numpy bf16 bits and torch)."""
+import numpy as np
+import torch
+
+from workloads import gen
+
+ATOL, RTOL = 1e-2, 2e-2          # the stated bar: |g - r| <= 1e-2 + 2e-2 |r|
+TIGHT_ATOL, TIGHT_RTOL = 1e-4, 4e-3  # what bf16 rounding of an fp32-accumulated result should meet
+
+
+def to_dev(bits):
+    return gen.bits_to_torch(bits).cuda()
+
+
+def to_f64(t):
+    """bf16 CUDA tensor -> float64 numpy (exact widening)."""
+    return gen.bf16_bits_to_f32(gen.torch_to_bits(t)).astype(np.float64)
+
+
+def assert_close(gpu_bf16, ref, what=""):
+    g = to_f64(gpu_bf16).reshape(ref.shape)
+    assert np.isfinite(g).all(), f"{what}: non-finite output"
+    err = np.abs(g - ref)
+    bound = ATOL + RTOL * np.abs(ref)
+    assert (err <= bound).all(), f"{what}: max err {err.max():.3e} beyond the stated tolerance"
+    tight = TIGHT_ATOL + TIGHT_RTOL * np.abs(ref)
+    assert (err <= tight).all(), f"{what}: max err {err.max():.3e} beyond bf16 rounding ({(err - tight).max():.3e} over)"
+    return err.max()
+
+
+def status_word():
+    return torch.zeros(1, dtype=torch.int32, device="cuda")
+
+
+def local_kv_split(kv_t):
+    """local cache tensor [..., C, 2, hd] (one layer: [B,H,C,2,hd]) -> K bits, V bits [B,H,C,hd]."""
+    bits = gen.torch_to_bits(kv_t)
+    return np.ascontiguousarray(bits[..., 0, :]), np.ascontiguousarray(bits[..., 1, :])
