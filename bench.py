@@ -1,0 +1,345 @@
+#!/usr/bin/env python
+"""Benchmark of the Block Transformer KV-cache attention path on B200.
+
+  python bench.py [--gpus N] [--steps K] [--warmup W] [--workload block_decode|token_decode|block_prefill]
+  python bench.py --impl reference ...      # times the CPU oracle instead (rank 0 only)
+
+Default workload: the block-decoder decode step (batch 256, 16 heads, head_dim 64, L_B = 4,
+2048-token context = 512 block-cache rows, 12 layers, each appending one row and attending).
+One step advances every sequence by one block = L_B tokens.  Prints ONE JSON line.
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import os
+import statistics
+import subprocess
+import sys
+import tempfile
+import time
+
+import numpy as np
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+sys.path.insert(0, ROOT)
+
+from workloads import configs, gen, traffic  # noqa: E402
+
+METRIC = "decode tokens/s (attention path)"
+FALLBACK_PEAKS = {"hbm_gbs": 6650.0, "bf16_tflops": 1590.0, "bf16_tflops_sustained": 1400.0}
+
+# DRAM traffic per launch of the dominant kernel, from the ncu captures summarised under profiles/
+# (dram__bytes_read.sum + dram__bytes_write.sum); None until a capture exists.
+NCU_TRAFFIC_BYTES = {"block_decode": None, "token_decode": None, "block_prefill": None}
+
+
+def peaks():
+    p = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    if os.path.exists(p):
+        with open(p) as f:
+            d = json.load(f)
+        d["_source"] = "measured"
+        return d
+    d = dict(FALLBACK_PEAKS)
+    d["_source"] = "fallback"
+    return d
+
+
+class ClockSampler:
+    """nvidia-smi clock / throttle-reason samples taken while the timed region runs."""
+    Q = ("index,clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.active,clocks_event_reasons.hw_slowdown,"
+         "clocks_event_reasons.hw_thermal_slowdown,clocks_event_reasons.sw_thermal_slowdown,"
+         "clocks_event_reasons.sw_power_cap")
+
+    def __init__(self, gpu_index: int):
+        self.gpu, self.proc, self.path = gpu_index, None, None
+
+    def start(self):
+        try:
+            fd, self.path = tempfile.mkstemp(suffix=".csv")
+            os.close(fd)
+            self.proc = subprocess.Popen(["nvidia-smi", f"--query-gpu={self.Q}", "--format=csv,noheader,nounits",
+                                          "-lms", "100", "-i", str(self.gpu)], stdout=open(self.path, "w"),
+                                         stderr=subprocess.DEVNULL)
+        except Exception:
+            self.proc = None
+
+    def stop(self):
+        out = {"sm_mhz": None, "sm_max_mhz": None, "reasons": [], "samples": 0}
+        if self.proc is None:
+            return out
+        self.proc.terminate()
+        try:
+            self.proc.wait(timeout=5)
+        except Exception:
+            self.proc.kill()
+        sm, mx, reasons = [], [], set()
+        try:
+            for line in open(self.path):
+                f = [x.strip() for x in line.split(",")]
+                if len(f) < 9:
+                    continue
+                try:
+                    sm.append(float(f[1]))
+                    mx.append(float(f[2]))
+                except ValueError:
+                    continue
+                for name, val in zip(("hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"), f[5:9]):
+                    if val.lower().startswith("active"):
+                        reasons.add(name)
+            os.unlink(self.path)
+        except Exception:
+            pass
+        if sm:
+            out.update(sm_mhz=statistics.median(sm), sm_max_mhz=max(mx), samples=len(sm))
+        out["reasons"] = sorted(reasons)
+        return out
+
+
+def dist_env():
+    return int(os.environ.get("RANK", 0)), int(os.environ.get("LOCAL_RANK", 0)), int(os.environ.get("WORLD_SIZE", 1))
+
+
+# ------------------------------------------------------------------------------------------ CPU oracle legs
+
+def oracle_block_decode_sample(w, n_seq, seed=None):
+    """Time the oracle on n_seq sequences of one layer of the block-decode step; returns
+    (seconds, sequences, layers) of the sample."""
+    import oracle
+    seed = w.seed if seed is None else seed
+    B, H, hd, N = n_seq, w.heads, w.head_dim, w.max_blocks
+    c = oracle.Cache(B, H, N, hd)
+    c.k[...] = gen.normal_bf16_bits(seed, 0, c.k.shape)
+    c.v[...] = gen.normal_bf16_bits(seed, 1, c.v.shape)
+    c.len[...] = w.ctx_blocks - 1
+    q, k, v = (gen.normal_bf16_bits(seed, 2 + i, (B, H, 1, hd)) for i in range(3))
+    oracle.lib()
+    t0 = time.perf_counter()
+    oracle.kv_append(c, k, v)
+    oracle.block_decode_attn(c, np.ascontiguousarray(q[:, :, 0]))
+    return time.perf_counter() - t0, n_seq, 1
+
+
+def cpu_baseline_block_decode(w, run):
+    """The oracle on the whole step (all sequences, all layers), fed the bytes the GPU run used:
+    each layer's cache is copied back to the host and handed to the oracle, which is timed alone."""
+    import oracle
+    oracle.lib()
+    B, H, hd, N = w.batch, w.heads, w.head_dim, w.max_blocks
+    secs = 0.0
+    for l in range(w.n_layers):
+        c = oracle.Cache(B, H, N, hd)
+        c.k[...] = gen.torch_to_bits(run.cache.k[l])
+        c.v[...] = gen.torch_to_bits(run.cache.v[l])
+        c.len[...] = w.ctx_blocks - 1
+        q, k, v = (gen.torch_to_bits(t[l]) for t in (run.q, run.k_new, run.v_new))
+        t0 = time.perf_counter()
+        oracle.kv_append(c, k, v)
+        oracle.block_decode_attn(c, np.ascontiguousarray(q[:, :, 0]))
+        secs += time.perf_counter() - t0
+    tokens = w.batch * w.block_len
+    return {"value": tokens / secs, "unit": "tokens/s", "cores": oracle.n_threads(), "kind": "oracle",
+            "sample": f"one full step: {w.batch} sequences x {w.n_layers} layers (append + attention, fp64), "
+                      f"{secs:.3f} s of oracle time, not scaled"}
+
+
+def run_reference(args):
+    """--impl reference: the CPU oracle, as it stands, on the machine's host cores."""
+    rank, _, world = dist_env()
+    if rank != 0:
+        return 0
+    import oracle
+    w = configs.BY_NAME[args.workload]
+    if args.workload != "block_decode":
+        print(json.dumps({"impl": "reference", "unavailable": "reference arm implemented for the block_decode workload only"}))
+        return 0
+    n_seq = 64
+    for _ in range(max(1, min(args.warmup, 2))):
+        oracle_block_decode_sample(w, n_seq)
+    times = []
+    for _ in range(args.steps):
+        secs, ns, nl = oracle_block_decode_sample(w, n_seq)
+        times.append(secs)
+    scale = (w.batch / n_seq) * w.n_layers
+    step_s = statistics.mean(times) * scale
+    tokens = w.batch * w.block_len
+    val = tokens / step_s
+    sample = f"per step: {n_seq} of {w.batch} sequences x 1 of {w.n_layers} layers, scaled x{scale:.0f}"
+    line = {"impl": "reference", "metric": METRIC, "value": val, "unit": "tokens/s", "n_gpus": args.gpus,
+            "steps": args.steps, "warmup": args.warmup, "ms_per_step": step_s * 1e3, "higher_is_better": True,
+            "scaling": "weak", "vs_baseline": None, "dtype": "f64", "data": "synthetic",
+            "config": workload_config(w, args.workload),
+            "cpu_baseline": {"value": val, "unit": "tokens/s", "cores": oracle.n_threads(), "kind": "oracle", "sample": sample},
+            "e2e": {"value": val, "unit": "tokens/s", "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0}}
+    print(json.dumps(line))
+    return 0
+
+
+def workload_config(w, name):
+    c = {"workload": name, "batch": w.batch, "heads": w.heads, "head_dim": w.head_dim, "block_len": w.block_len,
+         "prefix_len": w.prefix_len, "n_layers": w.n_layers}
+    if name == "block_decode":
+        c.update(workload="block_decode: BASELINE configs[1], per layer append 1 block row then attend over 512 rows",
+                 ctx_blocks=w.ctx_blocks, context_tokens=w.ctx_blocks * w.block_len,
+                 l2="no flush: 6.4 GB of KV per step, 537 MB per launch, L2 is 126 MB")
+    elif name == "token_decode":
+        c.update(workload="token_decode: BASELINE configs[2], fused reset+append+local attention, 12 launches per token step",
+                 l2="no flush: inputs rotate over a ring larger than L2")
+    elif name == "block_prefill":
+        c.update(workload="block_prefill: BASELINE configs[3], dense causal attention over 512 prompt blocks",
+                 prompt_blocks=w.prompt_blocks, l2="no flush: 3.2 GB of Q,K,V,out per step")
+    return c
+
+
+# ------------------------------------------------------------------------------------------ GPU arm
+
+def run_gpu(args):
+    import torch
+    import torch.distributed as dist
+
+    rank, local_rank, world = dist_env()
+    if not torch.cuda.is_available():
+        raise SystemExit("bench.py needs a CUDA device: the attention path has no CPU fallback")
+    torch.cuda.set_device(local_rank)
+    if world > 1:
+        dist.init_process_group("nccl", device_id=torch.device("cuda", local_rank))
+    import paper_2406_02657_b200 as bt  # noqa: F401  (loads libbt.so; raises if it cannot)
+    from paper_2406_02657_b200 import harness
+
+    w = configs.BY_NAME[args.workload]
+    reduced = {}
+    if args.batch:
+        reduced["batch"] = args.batch
+    if args.layers:
+        reduced["n_layers"] = args.layers
+    if reduced:  # a smaller copy of the workload, for profiler captures only
+        w = configs.scaled(w, **reduced)
+    fill = lambda tid, shape: gen.normal_bf16_device(w.seed + 17 * rank, tid, shape, device="cuda")
+    pk = peaks()
+
+    def barrier():
+        if world > 1:
+            dist.barrier()
+        torch.cuda.synchronize()
+
+    def timed(step_fn, pre_fn, steps, warmup):
+        """W untimed steps, then exactly K timed steps between barriers; returns ms per step (max over ranks)."""
+        for _ in range(warmup):
+            pre_fn()
+            step_fn()
+        barrier()
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        e0.record()
+        for _ in range(steps):
+            pre_fn()
+            step_fn()
+        e1.record()
+        barrier()
+        ms = e0.elapsed_time(e1) / steps
+        if world > 1:
+            t = torch.tensor([ms], device="cuda")
+            dist.all_reduce(t, op=dist.ReduceOp.MAX)
+            ms = t.item()
+        return ms
+
+    sampler = ClockSampler(local_rank)
+    kern_events = []
+    if args.workload == "block_decode":
+        run = harness.BlockDecodeStep(w, fill=fill)
+        tokens_per_step = w.batch * w.block_len
+        sampler.start()
+        ms = timed(lambda: run.step(kern_events), run.rewind, args.steps, args.warmup)
+        clocks = sampler.stop()
+        assert run.status.item() == 0 and (run.cache.len == w.ctx_blocks).all()
+        kern_events = kern_events[args.warmup * w.n_layers:]
+        ms_e2e = timed(run.step_host, run.rewind, args.steps, args.warmup)
+        h2d, d2h = run.host_bytes_per_step()
+        alg_bytes = traffic.block_decode_layer_bytes(w.batch, w.heads, w.head_dim, w.ctx_blocks, with_append=False)
+        dom = "block_decode_kernel"
+        launches = run.launches_per_step * args.steps
+        step_bytes = w.n_layers * traffic.block_decode_layer_bytes(w.batch, w.heads, w.head_dim, w.ctx_blocks, True)
+    elif args.workload == "token_decode":
+        run = harness.TokenDecodeRun(w, fill=fill)
+        tokens_per_step = w.batch
+        # a bench step = one block of L_B token steps so that every step does the same work
+        sampler.start()
+        ms_block = timed(lambda: [run.token_step() for _ in range(w.block_len)], lambda: None, args.steps, args.warmup)
+        clocks = sampler.stop()
+        ms = ms_block / w.block_len
+        ms_e2e, h2d, d2h = None, 0, 0
+        alg_bytes = sum(traffic.token_decode_layer_bytes(w.batch, w.heads, w.head_dim, j) for j in range(w.block_len)) / w.block_len
+        dom = "token_decode_kernel"
+        launches = run.launches_per_step * w.block_len * args.steps
+        step_bytes = w.n_layers * alg_bytes
+    else:
+        run = harness.PrefillRun(w, fill=fill)
+        tokens_per_step = w.batch * w.prompt_tokens
+        sampler.start()
+        ms = timed(lambda: run.step(kern_events), lambda: None, args.steps, args.warmup)
+        clocks = sampler.stop()
+        kern_events = kern_events[args.warmup * w.n_layers:]
+        ms_e2e, h2d, d2h = None, 0, 0
+        alg_bytes = traffic.prefill_layer_bytes(w.batch, w.heads, w.prompt_blocks, w.head_dim)
+        dom = "block_prefill_kernel"
+        launches = run.launches_per_step * args.steps
+        step_bytes = w.n_layers * alg_bytes
+
+    torch.cuda.synchronize()
+    if kern_events:
+        kern_ms = statistics.mean(a.elapsed_time(b) for a, b in kern_events)
+    else:
+        kern_ms = ms / run.launches_per_step
+    achieved = alg_bytes / (kern_ms * 1e-3) / 1e9
+    roof = {"bound": "hbm", "kernel": dom, "achieved": achieved, "peak": pk["hbm_gbs"], "unit": "GB/s",
+            "frac": achieved / pk["hbm_gbs"], "peak_source": f"of {pk['_source']} (copy bandwidth)",
+            "frac_of_8TBs_nominal": achieved / 8000.0, "kernel_ms": kern_ms, "algorithmic_bytes_per_launch": alg_bytes,
+            "traffic": NCU_TRAFFIC_BYTES.get(args.workload),
+            "step_GBs": step_bytes / (ms * 1e-3) / 1e9}
+    if args.workload == "block_prefill":
+        fl = traffic.prefill_layer_flops(w.batch, w.heads, w.prompt_blocks, w.head_dim)
+        roof["tensor_tflops"] = fl / (kern_ms * 1e-3) / 1e12
+        roof["tensor_frac_of_measured_burst"] = roof["tensor_tflops"] / pk["bf16_tflops"]
+
+    if rank != 0:
+        return 0
+    value = world * tokens_per_step / (ms * 1e-3)
+    line = {"metric": METRIC, "value": value, "unit": "tokens/s", "n_gpus": world, "steps": args.steps,
+            "warmup": args.warmup, "ms_per_step": ms, "higher_is_better": True, "scaling": "weak",
+            "vs_baseline": None, "dtype": "bf16", "accumulate": "f32", "data": "synthetic",
+            "config": workload_config(w, args.workload), "clocks": clocks, "gpu_launches": launches,
+            "roofline": roof}
+    if ms_e2e is not None:
+        line["e2e"] = {"value": world * tokens_per_step / (ms_e2e * 1e-3), "unit": "tokens/s", "ms_per_step": ms_e2e,
+                       "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h,
+                       "api": "bt_block_decode_step_host (pinned host q,k,v in; out back to host; cache resident)"}
+    if world == 1 and args.workload == "block_decode" and not args.no_cpu_baseline and not reduced:
+        line["cpu_baseline"] = cpu_baseline_block_decode(w, run)
+    if reduced:
+        line["reduced_case_not_a_bench_number"] = reduced
+    print(json.dumps(line))
+    if world > 1:
+        dist.destroy_process_group()
+    return 0
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=200)
+    ap.add_argument("--warmup", type=int, default=3)
+    ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
+    ap.add_argument("--workload", default="block_decode", choices=["block_decode", "token_decode", "block_prefill"])
+    ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--batch", type=int, default=0, help="override the batch (profiling a small case; not a bench number)")
+    ap.add_argument("--layers", type=int, default=0, help="override the layer count (profiling a small case)")
+    args = ap.parse_args()
+    if args.warmup < 3 and args.impl == "ours":
+        args.warmup = 3
+    if args.impl == "reference":
+        return run_reference(args)
+    return run_gpu(args)
+
+
+if __name__ == "__main__":
+    sys.exit(main())

@@ -1,0 +1,126 @@
+"""Synthetic drivers for the paper's serving workloads (section 3.2: prompts padded to one length,
+prefill-heavy 2048/128 and decode-heavy 128/2048): they own the device buffers and issue the
+library calls of one step.  No arithmetic of the method happens here.
+"""
+from __future__ import annotations
+
+import torch
+
+from . import binding as bt
+
+
+class BlockDecodeStep:
+    """One block-decoder decode step over all layers (section 2.3): per layer, append the new
+    block's K,V row, then attend causally over the whole block cache.
+
+    The caches are pre-filled to ``ctx_blocks - 1`` rows so that after the append every sequence
+    attends over ``ctx_blocks`` rows.  ``rewind()`` puts the lengths back so a step can be repeated.
+    """
+
+    def __init__(self, w, device="cuda", fill=None):
+        self.w, self.device = w, device
+        self.cfg = bt.make_config(w.batch, w.heads, w.head_dim, w.block_len, w.prefix_len, w.max_blocks, w.n_layers)
+        shape = (w.n_layers, w.batch, w.heads, w.max_blocks, w.head_dim)
+        if fill is None:
+            k = torch.zeros(shape, dtype=torch.bfloat16, device=device)
+            v = torch.zeros(shape, dtype=torch.bfloat16, device=device)
+        else:
+            k, v = fill(0, shape), fill(1, shape)
+        self.cache = bt.BlockCache(self.cfg, device, k=k, v=v)
+        self.len0 = torch.full((w.n_layers, w.batch), w.ctx_blocks - 1, dtype=torch.int32, device=device)
+        self.cache.len.copy_(self.len0)
+        io = (w.n_layers, w.batch, w.heads, 1, w.head_dim)
+        mk = (lambda tid: fill(tid, io)) if fill is not None else (lambda tid: torch.zeros(io, dtype=torch.bfloat16, device=device))
+        self.q, self.k_new, self.v_new = mk(2), mk(3), mk(4)
+        self.out = torch.empty(io, dtype=torch.bfloat16, device=device)
+        self.ws = bt.alloc_workspace(self.cfg, device)
+        self.status = torch.zeros(1, dtype=torch.int32, device=device)
+        # append + attention per layer, plus the merge pass when the row range is split
+        self.launches_per_step = w.n_layers * (2 + (1 if bt.bt_decode_splits(self.cfg) > 1 else 0))
+        self._host = None
+
+    def rewind(self):
+        self.cache.len.copy_(self.len0, non_blocking=True)
+
+    def step(self, attn_events=None):
+        """Enqueue one step.  attn_events: optional list receiving (start, stop) CUDA events around
+        each attention launch."""
+        for l in range(self.w.n_layers):
+            bt.bt_block_kv_append(self.cfg, self.cache, l, self.k_new[l], self.v_new[l], n_new=1, dev_status=self.status)
+            if attn_events is not None:
+                e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+                e0.record()
+            bt.bt_block_decode_attn(self.cfg, self.cache, l, self.q[l], self.out[l], self.ws, dev_status=self.status)
+            if attn_events is not None:
+                e1.record()
+                attn_events.append((e0, e1))
+
+    # ---- the same step driven from pinned host buffers through bt_block_decode_step_host
+    def _host_buffers(self):
+        if self._host is None:
+            pin = lambda t: t.cpu().pin_memory()
+            self._host = dict(q=pin(self.q), k=pin(self.k_new), v=pin(self.v_new), out=torch.empty_like(self.out, device="cpu").pin_memory(),
+                              qd=torch.empty_like(self.q), kd=torch.empty_like(self.k_new), vd=torch.empty_like(self.v_new))
+        return self._host
+
+    def host_bytes_per_step(self):
+        one = self.w.batch * self.w.heads * self.w.head_dim * 2
+        return 3 * one * self.w.n_layers, one * self.w.n_layers
+
+    def step_host(self):
+        h = self._host_buffers()
+        for l in range(self.w.n_layers):
+            bt.bt_block_decode_step_host(self.cfg, self.cache, l, h["q"][l], h["k"][l], h["v"][l], h["out"][l],
+                                         h["qd"][l], h["kd"][l], h["vd"][l], self.out[l], self.ws, dev_status=self.status)
+
+
+class TokenDecodeRun:
+    """Token-decoder steps over all layers (section 2.4): step j of a block resets (j == 0),
+    appends one row and attends over the local cache (prefix + tokens of the same block)."""
+
+    def __init__(self, w, device="cuda", fill=None, ring=8):
+        self.w, self.device = w, device
+        self.cfg = bt.make_config(w.batch, w.heads, w.head_dim, w.block_len, w.prefix_len, max(1, w.max_blocks), w.n_layers)
+        self.cache = bt.LocalCache(self.cfg, device)
+        io = (ring, w.n_layers, w.batch, w.heads, 1, w.head_dim)
+        mk = (lambda tid: fill(tid, io)) if fill is not None else (lambda tid: torch.zeros(io, dtype=torch.bfloat16, device=device))
+        self.q, self.k_new, self.v_new = mk(5), mk(6), mk(7)
+        self.out = torch.empty(io[1:], dtype=torch.bfloat16, device=device)
+        self.status = torch.zeros(1, dtype=torch.int32, device=device)
+        self.ring = ring
+        self.t = 0
+        self.launches_per_step = w.n_layers
+
+    def token_step(self):
+        """Token step t (prefix length 1: the prefix row is the first row of each block)."""
+        w = self.w
+        j = self.t % w.block_len
+        r = self.t % self.ring
+        for l in range(w.n_layers):
+            bt.bt_token_decode_attn(self.cfg, self.cache, l, self.q[r, l], self.k_new[r, l], self.v_new[r, l], self.out[l],
+                                    n_q=1, reset_first=(j == 0), dev_status=self.status)
+        self.t += 1
+
+
+class PrefillRun:
+    """Block-decoder prefill over all layers (sections 2.1, 2.3): dense causal attention over the
+    T prompt blocks, distinct Q, K, V, out per layer."""
+
+    def __init__(self, w, device="cuda", fill=None):
+        self.w = w
+        self.cfg = bt.make_config(w.batch, w.heads, w.head_dim, w.block_len, w.prefix_len, w.max_blocks, w.n_layers)
+        shape = (w.n_layers, w.batch, w.heads, w.prompt_blocks, w.head_dim)
+        mk = (lambda tid: fill(tid, shape)) if fill is not None else (lambda tid: torch.zeros(shape, dtype=torch.bfloat16, device=device))
+        self.q, self.k, self.v = mk(8), mk(9), mk(10)
+        self.out = torch.empty(shape, dtype=torch.bfloat16, device=device)
+        self.launches_per_step = w.n_layers
+
+    def step(self, events=None):
+        for l in range(self.w.n_layers):
+            if events is not None:
+                e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+                e0.record()
+            bt.bt_block_prefill_attn(self.cfg, self.q[l], self.k[l], self.v[l], self.out[l], n_blocks=self.w.prompt_blocks)
+            if events is not None:
+                e1.record()
+                events.append((e0, e1))
