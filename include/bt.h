@@ -66,6 +66,8 @@ typedef struct bt_config {
     int32_t decode_splits; /* 0: library chooses how many ways bt_block_decode_attn
                               splits the row range; >0: forced (tests, tuning)       */
     float softmax_scale;   /* 0 => 1/sqrt(head_dim)                                  */
+    int32_t prefill_plain; /* non-zero: bt_block_prefill_attn uses its CUDA-core kernel
+                              instead of the tensor-core one (testing; odd alignments) */
 } bt_config;
 
 /* Block-level KV cache (section 2.3): one row per block.
@@ -161,9 +163,14 @@ bt_status bt_token_decode_attn(const bt_config* cfg, bt_local_cache* cache, int 
  * q, out: [B][H][T][hd].  k, v: rows hd apart; (b,h) slab s starts s * kv_seq_stride rows
  * after the base, so kv_seq_stride = T for packed tensors and = N_max when k, v point at a
  * layer of a block cache that already holds the prompt's rows.  Requires kv_seq_stride >= T.
+ * Runs on the tensor cores (TMA-fed tcgen05 MMA, accumulators in tensor memory) when all four
+ * pointers are 16-byte aligned, else on a CUDA-core kernel.  Every wait inside the tensor-core
+ * kernel is bounded; one that runs out raises BT_DEV_TIMEOUT in *dev_status and leaves the
+ * affected output rows unwritten.
  */
 bt_status bt_block_prefill_attn(const bt_config* cfg, const void* q, const void* k, const void* v,
-                                int n_blocks, int64_t kv_seq_stride, void* out, void* stream);
+                                int n_blocks, int64_t kv_seq_stride, void* out, uint32_t* dev_status,
+                                void* stream);
 
 /*
  * One block-decoder decode step of one layer driven from HOST buffers (the same operations as

@@ -27,7 +27,8 @@ EXPORTS = [
 class bt_config(ctypes.Structure):
     _fields_ = [("batch", ctypes.c_int32), ("heads", ctypes.c_int32), ("head_dim", ctypes.c_int32),
                 ("block_len", ctypes.c_int32), ("prefix_len", ctypes.c_int32), ("max_blocks", ctypes.c_int32),
-                ("n_layers", ctypes.c_int32), ("decode_splits", ctypes.c_int32), ("softmax_scale", ctypes.c_float)]
+                ("n_layers", ctypes.c_int32), ("decode_splits", ctypes.c_int32), ("softmax_scale", ctypes.c_float),
+                ("prefill_plain", ctypes.c_int32)]
 
 
 class bt_block_cache(ctypes.Structure):
@@ -63,7 +64,7 @@ def _load() -> ctypes.CDLL:
     lib.bt_local_kv_reset.argtypes = [cfgp, ctypes.POINTER(bt_local_cache), i32, vp, vp]
     lib.bt_local_kv_append.argtypes = [cfgp, ctypes.POINTER(bt_local_cache), i32, vp, vp, i32, vp, vp]
     lib.bt_token_decode_attn.argtypes = [cfgp, ctypes.POINTER(bt_local_cache), i32, vp, vp, vp, i32, i32, vp, vp, vp, vp]
-    lib.bt_block_prefill_attn.argtypes = [cfgp, vp, vp, vp, i32, ctypes.c_int64, vp, vp]
+    lib.bt_block_prefill_attn.argtypes = [cfgp, vp, vp, vp, i32, ctypes.c_int64, vp, vp, vp]
     lib.bt_block_decode_step_host.argtypes = [cfgp, ctypes.POINTER(bt_block_cache), i32, vp, vp, vp, vp,
                                               vp, vp, vp, vp, vp, u64, vp, vp]
     for name in EXPORTS[4:]:
@@ -102,9 +103,9 @@ def _check(code: int, where: str):
 
 
 def make_config(batch, heads, head_dim, block_len, prefix_len, max_blocks, n_layers, decode_splits=0,
-                softmax_scale=0.0) -> bt_config:
+                softmax_scale=0.0, prefill_plain=0) -> bt_config:
     return bt_config(batch, heads, head_dim, block_len, prefix_len, max_blocks, n_layers, decode_splits,
-                     softmax_scale)
+                     softmax_scale, prefill_plain)
 
 
 class BlockCache:
@@ -179,11 +180,11 @@ def bt_token_decode_attn(cfg, cache: LocalCache, layer, q, k_new, v_new, out, n_
                                      _ptr(dev_status), _stream(stream)), "bt_token_decode_attn")
 
 
-def bt_block_prefill_attn(cfg, q, k, v, out, n_blocks=None, kv_seq_stride=None, stream=None):
+def bt_block_prefill_attn(cfg, q, k, v, out, n_blocks=None, kv_seq_stride=None, dev_status=None, stream=None):
     n_blocks = q.shape[2] if n_blocks is None else n_blocks
     kv_seq_stride = n_blocks if kv_seq_stride is None else kv_seq_stride
     _check(_lib.bt_block_prefill_attn(ctypes.byref(cfg), _ptr(q), _ptr(k), _ptr(v), n_blocks, kv_seq_stride,
-                                      _ptr(out), _stream(stream)), "bt_block_prefill_attn")
+                                      _ptr(out), _ptr(dev_status), _stream(stream)), "bt_block_prefill_attn")
 
 
 def bt_block_decode_step_host(cfg, cache: BlockCache, layer, q_host, k_new_host, v_new_host, out_host, q_dev, k_dev,

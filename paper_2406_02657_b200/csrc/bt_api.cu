@@ -205,7 +205,7 @@ bt_status bt_token_decode_attn(const bt_config* cfg, bt_local_cache* cache, int 
 }
 
 bt_status bt_block_prefill_attn(const bt_config* cfg, const void* q, const void* k, const void* v, int n_blocks,
-                                int64_t kv_seq_stride, void* out, void* stream)
+                                int64_t kv_seq_stride, void* out, uint32_t* dev_status, void* stream)
 {
     bt_status st = check_config(cfg, 0);
     if (st != BT_OK) return st;
@@ -222,6 +222,8 @@ bt_status bt_block_prefill_attn(const bt_config* cfg, const void* q, const void*
     a.T = n_blocks;
     a.kv_seq_stride = kv_seq_stride;
     a.scale_log2 = scale_log2(cfg);
+    if (!cfg->prefill_plain && bt::prefill_tc_supported(a))
+        return cuda_status(bt::launch_block_prefill_tc(a, dev_status, (cudaStream_t)stream));
     return cuda_status(bt::launch_block_prefill_simple(a, (cudaStream_t)stream));
 }
 

@@ -60,5 +60,8 @@ struct PrefillArgs {
 };
 // Plain CUDA-core kernel: any T, used for shapes the tensor-core kernel does not take.
 cudaError_t launch_block_prefill_simple(const PrefillArgs& a, cudaStream_t stream);
+// Tensor-core kernel (TMA + tcgen05 + TMEM): needs 16-byte aligned pointers.
+bool prefill_tc_supported(const PrefillArgs& a);
+cudaError_t launch_block_prefill_tc(const PrefillArgs& a, uint32_t* dev_status, cudaStream_t stream);
 
 }  // namespace bt

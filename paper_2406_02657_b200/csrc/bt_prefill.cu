@@ -1,0 +1,457 @@
+// Block-decoder prefill attention on the 5th-generation tensor cores (paper sections 2.1, 2.3:
+// the prefill stage processes all prompt blocks in parallel; causal over blocks).
+//
+// One CTA owns 128 query blocks of one (sequence, head) and walks the key/value blocks
+// 0 .. diagonal in tiles of 128:
+//   warp 4 (one lane): TMA producer - Q once, then K and V tiles into a 2-stage ring
+//   warp 5 (one lane): tcgen05.mma issuer - S = Q K^T into a double-buffered TMEM accumulator,
+//                      O += P V into a second TMEM accumulator
+//   warps 0-3        : softmax - each thread owns one query row (= one TMEM lane): row maximum,
+//                      exp2, bf16 P written to shared memory in the 128-byte-swizzled K-major
+//                      layout the MMA reads, running row sum; O is rescaled in TMEM only when the
+//                      row maximum grew by more than 2^8 (otherwise the old reference is kept,
+//                      which is exact because O and the row sum share the reference)
+// All waits are bounded: a wait that runs out raises BT_DEV_TIMEOUT and the CTA winds down.
+#include <cuda.h>
+
+#include "bt_common.cuh"
+#include "bt_kernels.h"
+
+namespace bt {
+namespace pf {
+
+constexpr int BM = 128;             // query rows per CTA
+constexpr int BN = 128;             // key/value rows per tile
+constexpr int kBoxBytes = 128 * 128;  // one TMA box: 128 rows x 64 bf16 (128 bytes, swizzled)
+constexpr int kThreads = 192;
+constexpr uint32_t kSpinLimit = 1u << 22;
+constexpr float kRescaleThreshold = 8.0f;  // log2 units
+
+// ---- barrier slots in shared memory
+enum { B_QFULL = 0, B_KFULL = 1, B_VFULL = 3, B_KVEMPTY = 5, B_SFULL = 7, B_SEMPTY = 9, B_PFULL = 11, B_PVDONE = 12, B_COUNT = 13 };
+
+__device__ __forceinline__ uint32_t smem_u32(const void* p) { return (uint32_t)__cvta_generic_to_shared(p); }
+
+__device__ __forceinline__ void mbar_init(uint32_t bar, uint32_t count)
+{
+    asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(bar), "r"(count) : "memory");
+}
+__device__ __forceinline__ void mbar_expect_tx(uint32_t bar, uint32_t bytes)
+{
+    asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(bar), "r"(bytes) : "memory");
+}
+__device__ __forceinline__ void mbar_arrive(uint32_t bar)
+{
+    asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(bar) : "memory");
+}
+__device__ __forceinline__ bool mbar_try_wait(uint32_t bar, uint32_t parity)
+{
+    uint32_t ok;
+    asm volatile(
+        "{\n\t.reg .pred p;\n\t"
+        "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
+        "selp.u32 %0, 1, 0, p;\n\t}"
+        : "=r"(ok)
+        : "r"(bar), "r"(parity)
+        : "memory");
+    return ok != 0;
+}
+// Bounded wait.  Returns false when the limit ran out or another thread of the CTA gave up.
+__device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatile int* abort_flag, uint32_t* dev_status)
+{
+    for (uint32_t it = 0; it < kSpinLimit; ++it) {
+        if (mbar_try_wait(bar, parity)) return true;
+        if ((it & 255u) == 255u && *abort_flag) return false;
+    }
+    *abort_flag = 1;
+    raise_status(dev_status, BT_DEV_TIMEOUT);
+    return false;
+}
+
+__device__ __forceinline__ void tma_load_3d(uint32_t dst, const CUtensorMap* map, uint32_t bar, int c0, int c1, int c2)
+{
+    asm volatile(
+        "cp.async.bulk.tensor.3d.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%3, %4, %5}], [%2];"
+        ::"r"(dst), "l"(map), "r"(bar), "r"(c0), "r"(c1), "r"(c2)
+        : "memory");
+}
+
+// Shared-memory matrix descriptor, 128-byte swizzle (layout type 2), descriptor version 1.
+__device__ __forceinline__ uint64_t make_desc(uint32_t saddr, uint32_t lbo_bytes, uint32_t sbo_bytes)
+{
+    uint64_t d = (uint64_t)((saddr & 0x3FFFFu) >> 4);
+    d |= (uint64_t)((lbo_bytes >> 4) & 0x3FFFu) << 16;
+    d |= (uint64_t)((sbo_bytes >> 4) & 0x3FFFu) << 32;
+    d |= (uint64_t)1 << 46;
+    d |= (uint64_t)2 << 61;
+    return d;
+}
+
+// Instruction descriptor: bf16 x bf16 -> fp32, A K-major, B K-major or MN-major.
+__host__ __device__ constexpr uint32_t make_idesc(int M, int N, bool b_mn_major)
+{
+    return (1u << 4) | (1u << 7) | (1u << 10) | ((b_mn_major ? 1u : 0u) << 16) | ((uint32_t)(N >> 3) << 17) |
+           ((uint32_t)(M >> 4) << 24);
+}
+
+__device__ __forceinline__ void mma_bf16(uint32_t tmem_d, uint64_t adesc, uint64_t bdesc, uint32_t idesc, uint32_t accumulate)
+{
+    asm volatile(
+        "{\n\t.reg .pred p;\n\t"
+        "setp.ne.b32 p, %4, 0;\n\t"
+        "tcgen05.mma.cta_group::1.kind::f16 [%0], %1, %2, %3, p;\n\t}"
+        ::"r"(tmem_d), "l"(adesc), "l"(bdesc), "r"(idesc), "r"(accumulate)
+        : "memory");
+}
+__device__ __forceinline__ void mma_commit(uint32_t bar)
+{
+    asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(bar) : "memory");
+}
+__device__ __forceinline__ void tc_fence_before() { asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory"); }
+__device__ __forceinline__ void tc_fence_after() { asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory"); }
+__device__ __forceinline__ void tmem_wait_ld() { asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory"); }
+__device__ __forceinline__ void tmem_wait_st() { asm volatile("tcgen05.wait::st.sync.aligned;" ::: "memory"); }
+
+// 32 consecutive fp32 columns of this thread's TMEM lane.
+__device__ __forceinline__ void tmem_ld32(uint32_t taddr, float (&v)[32])
+{
+    uint32_t r[32];
+    asm volatile(
+        "tcgen05.ld.sync.aligned.32x32b.x32.b32 "
+        "{%0, %1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15, "
+        "%16, %17, %18, %19, %20, %21, %22, %23, %24, %25, %26, %27, %28, %29, %30, %31}, [%32];"
+        : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]), "=r"(r[4]), "=r"(r[5]), "=r"(r[6]), "=r"(r[7]),
+          "=r"(r[8]), "=r"(r[9]), "=r"(r[10]), "=r"(r[11]), "=r"(r[12]), "=r"(r[13]), "=r"(r[14]), "=r"(r[15]),
+          "=r"(r[16]), "=r"(r[17]), "=r"(r[18]), "=r"(r[19]), "=r"(r[20]), "=r"(r[21]), "=r"(r[22]), "=r"(r[23]),
+          "=r"(r[24]), "=r"(r[25]), "=r"(r[26]), "=r"(r[27]), "=r"(r[28]), "=r"(r[29]), "=r"(r[30]), "=r"(r[31])
+        : "r"(taddr)
+        : "memory");
+    tmem_wait_ld();
+#pragma unroll
+    for (int i = 0; i < 32; ++i) v[i] = __uint_as_float(r[i]);
+}
+__device__ __forceinline__ void tmem_st32(uint32_t taddr, const float (&v)[32])
+{
+    asm volatile(
+        "tcgen05.st.sync.aligned.32x32b.x32.b32 [%0], "
+        "{%1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15, %16, "
+        "%17, %18, %19, %20, %21, %22, %23, %24, %25, %26, %27, %28, %29, %30, %31, %32};"
+        ::"r"(taddr),
+          "r"(__float_as_uint(v[0])), "r"(__float_as_uint(v[1])), "r"(__float_as_uint(v[2])), "r"(__float_as_uint(v[3])),
+          "r"(__float_as_uint(v[4])), "r"(__float_as_uint(v[5])), "r"(__float_as_uint(v[6])), "r"(__float_as_uint(v[7])),
+          "r"(__float_as_uint(v[8])), "r"(__float_as_uint(v[9])), "r"(__float_as_uint(v[10])), "r"(__float_as_uint(v[11])),
+          "r"(__float_as_uint(v[12])), "r"(__float_as_uint(v[13])), "r"(__float_as_uint(v[14])), "r"(__float_as_uint(v[15])),
+          "r"(__float_as_uint(v[16])), "r"(__float_as_uint(v[17])), "r"(__float_as_uint(v[18])), "r"(__float_as_uint(v[19])),
+          "r"(__float_as_uint(v[20])), "r"(__float_as_uint(v[21])), "r"(__float_as_uint(v[22])), "r"(__float_as_uint(v[23])),
+          "r"(__float_as_uint(v[24])), "r"(__float_as_uint(v[25])), "r"(__float_as_uint(v[26])), "r"(__float_as_uint(v[27])),
+          "r"(__float_as_uint(v[28])), "r"(__float_as_uint(v[29])), "r"(__float_as_uint(v[30])), "r"(__float_as_uint(v[31]))
+        : "memory");
+}
+
+struct Params {
+    void* out;
+    uint32_t* dev_status;
+    int T, n_qtiles;
+    float scale_log2;
+};
+
+template <int HD>
+constexpr int smem_bytes()
+{
+    // Q + 2 K stages + 2 V stages (HD/64 boxes each) + P (2 boxes) + barriers, plus 1024 to align
+    return 1024 + (HD / 64) * kBoxBytes * 5 + 2 * kBoxBytes + 256;
+}
+
+template <int HD>
+__global__ void __launch_bounds__(kThreads, 1)
+block_prefill_tc_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_constant__ CUtensorMap mapK,
+                        const __grid_constant__ CUtensorMap mapV, Params p)
+{
+    constexpr int NB = HD / 64;                 // TMA boxes per operand tile
+    constexpr uint32_t TILE_BYTES = NB * kBoxBytes;
+    constexpr uint32_t IDESC_S = make_idesc(BM, BN, false);
+    constexpr uint32_t IDESC_O = make_idesc(BM, HD, true);
+    constexpr uint32_t COL_S = 0, COL_O = 2 * BN;  // TMEM columns: S0 | S1 | O
+
+    extern __shared__ uint8_t smem_raw[];
+    const uint32_t base = (smem_u32(smem_raw) + 1023u) & ~1023u;
+    uint8_t* gen_base = smem_raw + (base - smem_u32(smem_raw));
+    const uint32_t sQ = base;
+    const uint32_t sK = sQ + TILE_BYTES;       // [2][TILE_BYTES]
+    const uint32_t sV = sK + 2 * TILE_BYTES;   // [2][TILE_BYTES]
+    const uint32_t sP = sV + 2 * TILE_BYTES;   // [2 boxes]
+    const uint32_t sBar = sP + 2 * kBoxBytes;  // B_COUNT x 8 bytes
+    uint8_t* gen_tail = gen_base + (sBar - base);
+    uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(gen_tail + B_COUNT * 8);
+    volatile int* abort_flag = reinterpret_cast<volatile int*>(gen_tail + B_COUNT * 8 + 8);
+    auto bar = [&](int i) { return sBar + 8u * i; };
+
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    const int bh = blockIdx.x / p.n_qtiles;
+    const int qt = p.n_qtiles - 1 - (blockIdx.x - bh * p.n_qtiles);  // heaviest query tiles first
+    const int n_kv = qt + 1;                                          // tiles 0 .. diagonal
+
+    if (threadIdx.x == 0) {
+        mbar_init(bar(B_QFULL), 1);
+        for (int s = 0; s < 2; ++s) {
+            mbar_init(bar(B_KFULL + s), 1);
+            mbar_init(bar(B_VFULL + s), 1);
+            mbar_init(bar(B_KVEMPTY + s), 1);
+            mbar_init(bar(B_SFULL + s), 1);
+            mbar_init(bar(B_SEMPTY + s), 128);
+        }
+        mbar_init(bar(B_PFULL), 128);
+        mbar_init(bar(B_PVDONE), 1);
+        *abort_flag = 0;
+        asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+    }
+    if (warp == 0) {  // allocate all 512 TMEM columns (S0, S1, O); this warp also frees them
+        asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(tmem_slot)), "r"(512u) : "memory");
+        asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
+    }
+    tc_fence_before();
+    __syncthreads();
+    tc_fence_after();
+    const uint32_t tmem = *tmem_slot;
+
+    if (warp == 4) {
+        // ------------------------------------------------------------------ TMA producer
+        if (lane == 0) {
+            asm volatile("prefetch.tensormap [%0];" ::"l"(&mapQ) : "memory");
+            asm volatile("prefetch.tensormap [%0];" ::"l"(&mapK) : "memory");
+            asm volatile("prefetch.tensormap [%0];" ::"l"(&mapV) : "memory");
+            mbar_expect_tx(bar(B_QFULL), TILE_BYTES);
+            for (int bx = 0; bx < NB; ++bx) tma_load_3d(sQ + bx * kBoxBytes, &mapQ, bar(B_QFULL), bx * 64, qt * BM, bh);
+            for (int j = 0; j < n_kv; ++j) {
+                const int st = j & 1;
+                if (j >= 2 && !mbar_wait(bar(B_KVEMPTY + st), ((j >> 1) - 1) & 1, abort_flag, p.dev_status)) break;
+                mbar_expect_tx(bar(B_KFULL + st), TILE_BYTES);
+                for (int bx = 0; bx < NB; ++bx)
+                    tma_load_3d(sK + st * TILE_BYTES + bx * kBoxBytes, &mapK, bar(B_KFULL + st), bx * 64, j * BN, bh);
+                mbar_expect_tx(bar(B_VFULL + st), TILE_BYTES);
+                for (int bx = 0; bx < NB; ++bx)
+                    tma_load_3d(sV + st * TILE_BYTES + bx * kBoxBytes, &mapV, bar(B_VFULL + st), bx * 64, j * BN, bh);
+            }
+        }
+    } else if (warp == 5) {
+        // ------------------------------------------------------------------ MMA issuer
+        if (lane == 0) {
+            bool ok = mbar_wait(bar(B_QFULL), 0, abort_flag, p.dev_status);
+            auto issue_pv = [&](int t) -> bool {
+                const int st = t & 1;
+                if (!mbar_wait(bar(B_PFULL), t & 1, abort_flag, p.dev_status)) return false;
+                if (!mbar_wait(bar(B_VFULL + st), (t >> 1) & 1, abort_flag, p.dev_status)) return false;
+                tc_fence_after();
+#pragma unroll
+                for (int kk = 0; kk < BN / 16; ++kk) {
+                    // A = P, K-major: 16 kv columns = 32 bytes inside the swizzled 128-byte row
+                    const uint64_t a = make_desc(sP + (kk >> 2) * kBoxBytes + (kk & 3) * 32, 16, 1024);
+                    // B = V, MN-major: 16 kv rows = 2048 bytes; next 64 head dims one box further
+                    const uint64_t b = make_desc(sV + st * TILE_BYTES + kk * 2048, kBoxBytes, 1024);
+                    mma_bf16(tmem + COL_O, a, b, IDESC_O, (t > 0 || kk > 0) ? 1u : 0u);
+                }
+                mma_commit(bar(B_KVEMPTY + st));
+                mma_commit(bar(B_PVDONE));
+                return true;
+            };
+            for (int j = 0; ok && j < n_kv; ++j) {
+                const int st = j & 1;
+                ok = mbar_wait(bar(B_KFULL + st), (j >> 1) & 1, abort_flag, p.dev_status);
+                if (ok && j >= 2) ok = mbar_wait(bar(B_SEMPTY + st), ((j >> 1) - 1) & 1, abort_flag, p.dev_status);
+                if (!ok) break;
+                tc_fence_after();
+#pragma unroll
+                for (int kk = 0; kk < HD / 16; ++kk) {
+                    const uint32_t off = (kk >> 2) * kBoxBytes + (kk & 3) * 32;
+                    const uint64_t a = make_desc(sQ + off, 16, 1024);
+                    const uint64_t b = make_desc(sK + st * TILE_BYTES + off, 16, 1024);
+                    mma_bf16(tmem + COL_S + st * BN, a, b, IDESC_S, kk > 0 ? 1u : 0u);
+                }
+                mma_commit(bar(B_SFULL + st));
+                if (j >= 1) ok = issue_pv(j - 1);
+            }
+            if (ok) issue_pv(n_kv - 1);
+        }
+    } else {
+        // ------------------------------------------------------------------ softmax: thread = query row
+        const int row = threadIdx.x;                       // TMEM lane
+        const int grow = qt * BM + row;                    // query block index within the sequence
+        const uint32_t lane_base = tmem + ((uint32_t)(warp * 32) << 16);
+        float m_ref = kNegInf, l = 0.f;
+        bool ok = true;
+        for (int j = 0; j < n_kv; ++j) {
+            const int st = j & 1;
+            const bool diag = (j == qt);
+            ok = mbar_wait(bar(B_SFULL + st), (j >> 1) & 1, abort_flag, p.dev_status);
+            if (!ok) break;
+            tc_fence_after();
+            const uint32_t s_addr = lane_base + COL_S + st * BN;
+            // pass 1: row maximum over the allowed columns
+            float mx = kNegInf;
+#pragma unroll 1
+            for (int c0 = 0; c0 < BN; c0 += 32) {
+                float v[32];
+                tmem_ld32(s_addr + c0, v);
+#pragma unroll
+                for (int i = 0; i < 32; ++i)
+                    if (!diag || c0 + i <= row) mx = fmaxf(mx, v[i]);
+            }
+            mx *= p.scale_log2;
+            float factor = 1.f;
+            const bool grow_ref = mx > m_ref + kRescaleThreshold;  // first tile: m_ref = -inf
+            if (grow_ref) {
+                factor = (m_ref == kNegInf) ? 0.f : ex2(m_ref - mx);
+                m_ref = mx;
+            }
+            if (j > 0) {
+                ok = mbar_wait(bar(B_PVDONE), (j - 1) & 1, abort_flag, p.dev_status);  // P buffer free, O settled
+                if (!ok) break;
+                tc_fence_after();
+                if (__any_sync(0xffffffffu, grow_ref)) {
+#pragma unroll 1
+                    for (int c0 = 0; c0 < HD; c0 += 32) {
+                        float o[32];
+                        tmem_ld32(lane_base + COL_O + c0, o);
+#pragma unroll
+                        for (int i = 0; i < 32; ++i) o[i] *= factor;
+                        tmem_st32(lane_base + COL_O + c0, o);
+                    }
+                    tmem_wait_st();
+                }
+                l *= factor;
+            }
+            // pass 2: P = 2^(s*scale - m_ref), bf16, into the swizzled K-major tile; row sum of what the MMA will see
+#pragma unroll 1
+            for (int c0 = 0; c0 < BN; c0 += 32) {
+                float v[32];
+                tmem_ld32(s_addr + c0, v);
+                uint32_t packed[16];
+#pragma unroll
+                for (int i = 0; i < 32; i += 2) {
+                    float p0 = (!diag || c0 + i <= row) ? ex2(fmaf(v[i], p.scale_log2, -m_ref)) : 0.f;
+                    float p1 = (!diag || c0 + i + 1 <= row) ? ex2(fmaf(v[i + 1], p.scale_log2, -m_ref)) : 0.f;
+                    __nv_bfloat162 pk = __floats2bfloat162_rn(p0, p1);
+                    uint32_t w = *reinterpret_cast<uint32_t*>(&pk);
+                    packed[i >> 1] = w;
+                    l += bf_lo(w) + bf_hi(w);
+                }
+                const uint32_t box = sP + (c0 >> 6) * kBoxBytes + row * 128;
+#pragma unroll
+                for (int q4 = 0; q4 < 4; ++q4) {
+                    const uint32_t chunk = (uint32_t)(((c0 & 63) >> 3) + q4) ^ (uint32_t)(row & 7);
+                    asm volatile("st.shared.v4.u32 [%0], {%1, %2, %3, %4};" ::"r"(box + chunk * 16), "r"(packed[4 * q4]),
+                                 "r"(packed[4 * q4 + 1]), "r"(packed[4 * q4 + 2]), "r"(packed[4 * q4 + 3])
+                                 : "memory");
+                }
+            }
+            tc_fence_before();
+            asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+            mbar_arrive(bar(B_SEMPTY + st));
+            mbar_arrive(bar(B_PFULL));
+        }
+        if (ok) ok = mbar_wait(bar(B_PVDONE), (n_kv - 1) & 1, abort_flag, p.dev_status);
+        if (ok) {
+            tc_fence_after();
+            const float inv = l > 0.f ? 1.f / l : 0.f;
+            bf16* orow = reinterpret_cast<bf16*>(p.out) + ((size_t)bh * p.T + grow) * HD;
+#pragma unroll 1
+            for (int c0 = 0; c0 < HD; c0 += 32) {
+                float o[32];
+                tmem_ld32(lane_base + COL_O + c0, o);
+                if (grow < p.T) {
+#pragma unroll
+                    for (int q8 = 0; q8 < 4; ++q8) {
+                        float f[8];
+#pragma unroll
+                        for (int i = 0; i < 8; ++i) f[i] = o[q8 * 8 + i] * inv;
+                        *reinterpret_cast<uint4*>(orow + c0 + q8 * 8) = pack8(f);
+                    }
+                }
+            }
+        }
+    }
+
+    tc_fence_before();
+    __syncthreads();
+    if (warp == 0) {
+        tc_fence_after();
+        asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem), "r"(512u) : "memory");
+    }
+}
+
+// ---- host side: tensor maps through the driver entry point (no link-time dependency on libcuda)
+using EncodeFn = CUresult (*)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*, const cuuint64_t*,
+                              const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave, CUtensorMapSwizzle,
+                              CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
+
+static EncodeFn encode_fn()
+{
+    static EncodeFn fn = nullptr;
+    static bool tried = false;
+    if (!tried) {
+        tried = true;
+        void* f = nullptr;
+        cudaDriverEntryPointQueryResult q;
+        if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &f, cudaEnableDefault, &q) == cudaSuccess &&
+            q == cudaDriverEntryPointSuccess)
+            fn = reinterpret_cast<EncodeFn>(f);
+    }
+    return fn;
+}
+
+// [slabs][rows][hd] bf16 with `stride_rows` rows between slabs; box = 64 x 128 x 1, 128-byte swizzle,
+// rows past `rows` read as zeros.
+static bool make_map(CUtensorMap* m, const void* ptr, int hd, int rows, long long stride_rows, long long slabs)
+{
+    EncodeFn fn = encode_fn();
+    if (!fn) return false;
+    cuuint64_t dims[3] = {(cuuint64_t)hd, (cuuint64_t)rows, (cuuint64_t)slabs};
+    cuuint64_t strides[2] = {(cuuint64_t)hd * 2, (cuuint64_t)stride_rows * hd * 2};
+    cuuint32_t box[3] = {64, 128, 1};
+    cuuint32_t estr[3] = {1, 1, 1};
+    return fn(m, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 3, const_cast<void*>(ptr), dims, strides, box, estr,
+              CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+              CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
+}
+
+template <int HD>
+static cudaError_t launch_t(const PrefillArgs& a, uint32_t* dev_status, cudaStream_t stream)
+{
+    static bool attr_set = false;
+    if (!attr_set) {
+        cudaError_t e = cudaFuncSetAttribute(block_prefill_tc_kernel<HD>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                             smem_bytes<HD>());
+        if (e != cudaSuccess) return e;
+        attr_set = true;
+    }
+    const long long slabs = (long long)a.B * a.H;
+    CUtensorMap mq, mk, mv;
+    if (!make_map(&mq, a.q, HD, a.T, a.T, slabs) || !make_map(&mk, a.k, HD, a.T, a.kv_seq_stride, slabs) ||
+        !make_map(&mv, a.v, HD, a.T, a.kv_seq_stride, slabs))
+        return cudaErrorInvalidValue;
+    Params p;
+    p.out = a.out;
+    p.dev_status = dev_status;
+    p.T = a.T;
+    p.n_qtiles = (a.T + BM - 1) / BM;
+    p.scale_log2 = a.scale_log2;
+    const long long ctas = slabs * p.n_qtiles;
+    if (ctas > 0x7fffffffLL) return cudaErrorInvalidConfiguration;
+    block_prefill_tc_kernel<HD><<<(unsigned)ctas, kThreads, smem_bytes<HD>(), stream>>>(mq, mk, mv, p);
+    return cudaGetLastError();
+}
+
+}  // namespace pf
+
+bool prefill_tc_supported(const PrefillArgs& a)
+{
+    auto al = [](const void* p) { return (reinterpret_cast<uintptr_t>(p) & 15u) == 0; };
+    return (a.hd == 64 || a.hd == 128) && al(a.q) && al(a.k) && al(a.v) && al(a.out) && pf::encode_fn() != nullptr;
+}
+
+cudaError_t launch_block_prefill_tc(const PrefillArgs& a, uint32_t* dev_status, cudaStream_t stream)
+{
+    return a.hd == 64 ? pf::launch_t<64>(a, dev_status, stream) : pf::launch_t<128>(a, dev_status, stream);
+}
+
+}  // namespace bt

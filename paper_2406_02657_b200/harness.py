@@ -101,6 +101,24 @@ class TokenDecodeRun:
                                     n_q=1, reset_first=(j == 0), dev_status=self.status)
         self.t += 1
 
+    def capture(self, n_steps=None):
+        """Capture n_steps consecutive token steps (default: one pass over the input ring, a whole
+        number of blocks) into a CUDA graph; replay() then advances the run by that many steps."""
+        n_steps = self.ring if n_steps is None else n_steps
+        assert n_steps % self.w.block_len == 0 and self.t % self.w.block_len == 0
+        self.token_step()  # make sure nothing lazy (module load) happens inside the capture
+        self.t -= 1
+        torch.cuda.synchronize()
+        self.graph = torch.cuda.CUDAGraph()
+        with torch.cuda.graph(self.graph):
+            for _ in range(n_steps):
+                self.token_step()
+        self.graph_steps = n_steps
+        return n_steps
+
+    def replay(self):
+        self.graph.replay()
+
 
 class PrefillRun:
     """Block-decoder prefill over all layers (sections 2.1, 2.3): dense causal attention over the

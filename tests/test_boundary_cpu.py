@@ -82,9 +82,9 @@ def test_host_detectable_errors_return_before_launch(bt):
     assert L.bt_token_decode_attn(ref(cfg), ref(lc), 0, fake, fake, fake, 0, 0, None, fake, None, None) == bt.BT_ERR_SHAPE
     assert L.bt_token_decode_attn(ref(cfg), ref(lc), 0, fake, fake, fake, 1, 0, None, None, None, None) == bt.BT_ERR_NULL
     # prefill
-    assert L.bt_block_prefill_attn(ref(cfg), fake, fake, fake, 0, 8, fake, None) == bt.BT_ERR_SHAPE
-    assert L.bt_block_prefill_attn(ref(cfg), fake, fake, fake, 16, 8, fake, None) == bt.BT_ERR_SHAPE
-    assert L.bt_block_prefill_attn(ref(cfg), fake, None, fake, 8, 8, fake, None) == bt.BT_ERR_NULL
+    assert L.bt_block_prefill_attn(ref(cfg), fake, fake, fake, 0, 8, fake, None, None) == bt.BT_ERR_SHAPE
+    assert L.bt_block_prefill_attn(ref(cfg), fake, fake, fake, 16, 8, fake, None, None) == bt.BT_ERR_SHAPE
+    assert L.bt_block_prefill_attn(ref(cfg), fake, None, fake, 8, 8, fake, None, None) == bt.BT_ERR_NULL
     # host-driven step
     assert L.bt_block_decode_step_host(ref(cfg), ref(bc), 0, None, fake, fake, fake, fake, fake, fake, fake,
                                        None, 0, None, None) == bt.BT_ERR_NULL

@@ -74,7 +74,7 @@ def test_tiny_prefill_packed_and_from_cache(bt):
     ref = oracle.block_prefill_attn(q, k, v)
     out = torch.empty((B, H, T, hd), dtype=torch.bfloat16, device="cuda")
     bt.bt_block_prefill_attn(cfg, to_dev(q), to_dev(k), to_dev(v), out)
-    assert_close(out, ref, "prefill packed")
+    assert_close(out, ref, "prefill packed", p_bf16=True)
     # bulk append of the prompt's rows, then prefill reading K,V in place from the cache
     cache = bt.BlockCache(cfg)
     st = status_word()
@@ -266,19 +266,41 @@ def test_l_b_one_block_decoder_is_vanilla_causal_attention(bt):
 
 # ------------------------------------------------------------------ prefill: tiles, diagonal, strides
 
-@pytest.mark.parametrize("hd,T,B,H", [(128, 128, 2, 2), (128, 300, 1, 3), (64, 257, 2, 2), (128, 512, 1, 2), (64, 33, 3, 1)])
-def test_block_prefill_shapes(bt, hd, T, B, H):
-    cfg = bt.make_config(B, H, hd, 4, 1, T, 1)
+@pytest.mark.parametrize("plain", [0, 1])
+@pytest.mark.parametrize("hd,T,B,H", [(128, 128, 2, 2), (128, 300, 1, 3), (64, 257, 2, 2), (128, 512, 1, 2), (64, 33, 3, 1),
+                                      (128, 1, 1, 1), (64, 640, 1, 2), (128, 1024, 1, 1)])
+def test_block_prefill_shapes(bt, hd, T, B, H, plain):
+    cfg = bt.make_config(B, H, hd, 4, 1, T, 1, prefill_plain=plain)
     q, k, v = (rnd(100 + T, i, (B, H, T, hd)) for i in range(3))
+    out = torch.full((B, H, T, hd), 9.0, dtype=torch.bfloat16, device="cuda")
+    st = status_word()
+    bt.bt_block_prefill_attn(cfg, to_dev(q), to_dev(k), to_dev(v), out, dev_status=st)
+    assert st.item() == 0
+    assert_close(out, oracle.block_prefill_attn(q, k, v), f"prefill T={T} hd={hd} plain={plain}", p_bf16=not plain)
+
+
+@pytest.mark.parametrize("plain", [0, 1])
+def test_block_prefill_reads_cache_in_place_and_ignores_rows_past_T(bt, plain):
+    """K, V taken in place from a block cache (stride N_max > T); rows past T hold NaN and must not matter."""
+    B, H, hd, T, N = 2, 3, 128, 200, 320
+    cfg = bt.make_config(B, H, hd, 4, 1, N, 1, prefill_plain=plain)
+    q = rnd(120, 0, (B, H, T, hd))
+    k, v = rnd(120, 1, (B, H, N, hd)), rnd(120, 2, (B, H, N, hd))
+    ref = oracle.block_prefill_attn(q, k, v, kv_seq_stride=N)
+    k[:, :, T:] = 0x7FC0
+    v[:, :, T:] = 0x7FC0
     out = torch.empty((B, H, T, hd), dtype=torch.bfloat16, device="cuda")
-    bt.bt_block_prefill_attn(cfg, to_dev(q), to_dev(k), to_dev(v), out)
-    assert_close(out, oracle.block_prefill_attn(q, k, v), f"prefill T={T} hd={hd}")
+    st = status_word()
+    bt.bt_block_prefill_attn(cfg, to_dev(q), to_dev(k), to_dev(v), out, n_blocks=T, kv_seq_stride=N, dev_status=st)
+    assert st.item() == 0
+    assert_close(out, ref, f"prefill from cache plain={plain}", p_bf16=not plain)
 
 
-def test_block_prefill_spikes_on_and_next_to_the_diagonal(bt):
+@pytest.mark.parametrize("plain", [0, 1])
+def test_block_prefill_spikes_on_and_next_to_the_diagonal(bt, plain):
     """A dominant key at block j must take over every query t >= j and no query t < j."""
     B, H, hd, T = 1, 1, 128, 384
-    cfg = bt.make_config(B, H, hd, 4, 1, T, 1)
+    cfg = bt.make_config(B, H, hd, 4, 1, T, 1, prefill_plain=plain)
     q = gen.f32_to_bf16_bits(np.full((B, H, T, hd), 1.5, np.float32))
     k, v = rnd(110, 1, (B, H, T, hd)), rnd(110, 2, (B, H, T, hd))
     spike_v = gen.f32_to_bf16_bits((np.arange(hd) - 60.0).astype(np.float32))
@@ -288,7 +310,23 @@ def test_block_prefill_spikes_on_and_next_to_the_diagonal(bt):
         kk[0, 0, j] = gen.f32_to_bf16_bits(np.full(hd, 8.0, np.float32))
         vv[0, 0, j] = spike_v
         bt.bt_block_prefill_attn(cfg, to_dev(q), to_dev(kk), to_dev(vv), out)
-        assert_close(out, oracle.block_prefill_attn(q, kk, vv), f"diagonal spike at {j}")
+        assert_close(out, oracle.block_prefill_attn(q, kk, vv), f"diagonal spike at {j}", p_bf16=not plain)
         got = to_f64(out)[0, 0]
         hit = np.abs(got - gen.bf16_bits_to_f32(spike_v)).max(axis=1) < 0.3
         assert hit[j:].all() and not hit[:j].any(), f"causal boundary wrong around block {j}"
+
+
+def test_block_prefill_late_large_keys_force_a_rescale(bt):
+    """Keys that grow along the sequence push the running row maximum up by far more than the
+    lazy-rescale threshold in every later tile, so the accumulator rescale path is exercised."""
+    B, H, hd, T = 1, 2, 128, 512
+    cfg = bt.make_config(B, H, hd, 4, 1, T, 1)
+    q = gen.f32_to_bf16_bits(np.abs(gen.bf16_bits_to_f32(rnd(130, 0, (B, H, T, hd)))))
+    ramp = (1.0 + np.arange(T, dtype=np.float32) / 16.0)[None, None, :, None]
+    k = gen.f32_to_bf16_bits(np.abs(gen.bf16_bits_to_f32(rnd(130, 1, (B, H, T, hd)))) * ramp)
+    v = rnd(130, 2, (B, H, T, hd))
+    out = torch.empty((B, H, T, hd), dtype=torch.bfloat16, device="cuda")
+    st = status_word()
+    bt.bt_block_prefill_attn(cfg, to_dev(q), to_dev(k), to_dev(v), out, dev_status=st)
+    assert st.item() == 0
+    assert_close(out, oracle.block_prefill_attn(q, k, v), "prefill with growing keys", p_bf16=True)

@@ -17,13 +17,20 @@ def to_f64(t):
     return gen.bf16_bits_to_f32(gen.torch_to_bits(t)).astype(np.float64)
 
 
-def assert_close(gpu_bf16, ref, what=""):
+# The tensor-core prefill feeds the softmax numerators to the second product as bf16 (8-bit
+# mantissa, like K and V).  Each term p_j v_j then carries up to 2^-9 relative error, so the
+# output error is bounded by 2^-9 * sum_j p_j |v_j| <= 2^-9 * max|v| (about 5 for N(0,1) values),
+# independent of how small the output itself is, plus the bf16 rounding of the output.
+P_BF16_ATOL, P_BF16_RTOL = 6e-3, 8e-3
+
+
+def assert_close(gpu_bf16, ref, what="", p_bf16=False):
     g = to_f64(gpu_bf16).reshape(ref.shape)
     assert np.isfinite(g).all(), f"{what}: non-finite output"
     err = np.abs(g - ref)
     bound = ATOL + RTOL * np.abs(ref)
     assert (err <= bound).all(), f"{what}: max err {err.max():.3e} beyond the stated tolerance"
-    tight = TIGHT_ATOL + TIGHT_RTOL * np.abs(ref)
+    tight = (P_BF16_ATOL + P_BF16_RTOL * np.abs(ref)) if p_bf16 else (TIGHT_ATOL + TIGHT_RTOL * np.abs(ref))
     assert (err <= tight).all(), f"{what}: max err {err.max():.3e} beyond bf16 rounding ({(err - tight).max():.3e} over)"
     return err.max()
 
