@@ -21,8 +21,15 @@ __device__ __forceinline__ void add_row(SoftmaxState& st, float s, const uint4& 
     st.m = mn;
 }
 
+#ifndef BT_TOK_MINBLOCKS
+#define BT_TOK_MINBLOCKS 3
+#endif
+#ifndef BT_TOK_THREADS
+#define BT_TOK_THREADS 256
+#endif
+
 template <int HD>
-__global__ void __launch_bounds__(256) token_decode_kernel(TokenArgs a, int seqs_per_cta, int threads_per_seq)
+__global__ void __launch_bounds__(256, BT_TOK_MINBLOCKS) token_decode_kernel(TokenArgs a, int seqs_per_cta, int threads_per_seq)
 {
     constexpr int LPR = RowGeo<HD>::LPR;
     const int tid = threadIdx.x;
@@ -32,18 +39,8 @@ __global__ void __launch_bounds__(256) token_decode_kernel(TokenArgs a, int seqs
     const int b = blockIdx.x * seqs_per_cta + sic;
     const bool active = sic < seqs_per_cta && b < a.B;
 
-    int len_old = 0;
-    if (active) {
-        const bool rst = a.reset_mask ? (a.reset_mask[b] != 0) : (a.reset_first != 0);
-        len_old = rst ? 0 : a.len[b];
-    }
-    __syncthreads();  // every head has read len[b] before the leader overwrites it
-
     const bool appended = a.k_new != nullptr;
-    const bool overflow = appended && (len_old < 0 || len_old + a.n_q > a.cap);
-    if (len_old < 0) len_old = 0;
-    if (len_old > a.cap) len_old = a.cap;
-
+    const bool fast = a.n_q == 1 && appended;
     const size_t slab = active ? (size_t)b * a.H + h : 0;
     bf16* cache = reinterpret_cast<bf16*>(a.kv) + slab * a.cap * 2 * HD + sub * 8;  // row r: K at +r*2*HD, V at +(r*2+1)*HD
     const bf16* qp = reinterpret_cast<const bf16*>(a.q) + slab * a.n_q * HD + sub * 8;
@@ -51,15 +48,27 @@ __global__ void __launch_bounds__(256) token_decode_kernel(TokenArgs a, int seqs
     const bf16* vp = reinterpret_cast<const bf16*>(a.v_new) + slab * a.n_q * HD + sub * 8;
     bf16* op = reinterpret_cast<bf16*>(a.out) + slab * a.n_q * HD + sub * 8;
 
-    if (a.n_q == 1 && appended) {
+    // the new row does not depend on the length: get it in flight before the length arrives
+    uint4 qr = make_uint4(0, 0, 0, 0), kr = qr, vr = qr;
+    if (fast && active) {
+        qr = ld_stream(qp);
+        kr = ld_stream(kp);
+        vr = ld_stream(vp);
+    }
+    int len_old = 0;
+    if (active) {
+        const bool rst = a.reset_mask ? (a.reset_mask[b] != 0) : (a.reset_first != 0);
+        len_old = rst ? 0 : a.len[b];
+    }
+    __syncthreads();  // every head has read len[b] before the leader overwrites it
+
+    const bool overflow = appended && (len_old < 0 || len_old + a.n_q > a.cap);
+    if (len_old < 0) len_old = 0;
+    if (len_old > a.cap) len_old = a.cap;
+
+    if (fast) {
         // token step: the new row stays in registers, the cached rows are read once
-        uint4 qr = make_uint4(0, 0, 0, 0), kr = qr, vr = qr;
         const int n_old = (active && !overflow) ? len_old : 0;
-        if (active) {
-            qr = ld_stream(qp);
-            kr = ld_stream(kp);
-            vr = ld_stream(vp);
-        }
         float qf[8];
         unpack8(qr, qf);
 #pragma unroll
@@ -137,11 +146,217 @@ __global__ void __launch_bounds__(256) token_decode_kernel(TokenArgs a, int seqs
     }
 }
 
+// ---------------------------------------------------------------------------------------
+// Pipelined token step (n_q = 1 with append: the per-token hot path).  The step is a stream of
+// tiny independent problems whose only serial hop is "read the length, then fetch that many
+// rows".  A persistent CTA walks groups of whole sequences and keeps kDepth groups in flight:
+// each thread copies the 16-byte pieces it will need (q, k_new, v_new and the cached rows below
+// the length) with cp.async into shared-memory slots that only it reads back, so no barrier is
+// needed for the data, and the lengths are fetched one group further ahead.  The one barrier per
+// group orders "every head has read len[b]" before "the leader writes the new len[b]".
+__device__ __forceinline__ void cp_async16(uint32_t dst, const void* src)
+{
+    asm volatile("cp.async.cg.shared.global [%0], [%1], 16;" ::"r"(dst), "l"(src) : "memory");
+}
+__device__ __forceinline__ void cp_async_commit() { asm volatile("cp.async.commit_group;" ::: "memory"); }
+template <int N>
+__device__ __forceinline__ void cp_async_wait() { asm volatile("cp.async.wait_group %0;" ::"n"(N) : "memory"); }
+
+constexpr int kTokThreads = 256;
+
+template <int HD, int kDepth, int kMaxRows, int kMinBlocks>
+__global__ void __launch_bounds__(kTokThreads, kMinBlocks)
+token_step_pipelined_kernel(TokenArgs a, int seqs_per_cta, int threads_per_seq)
+{
+    constexpr int max_rows = kMaxRows;
+    constexpr int LPR = RowGeo<HD>::LPR;
+    constexpr int kStages = kDepth + 1;
+    extern __shared__ uint4 slots_mem[];  // [kStages][3 + 2*max_rows][kTokThreads]
+    constexpr int n_slots = 3 + 2 * max_rows;
+    const int tid = threadIdx.x;
+    const int sic = tid / threads_per_seq;
+    const int within = tid - sic * threads_per_seq;
+    const int h = within / LPR, sub = within % LPR;
+    const bool lane_used = sic < seqs_per_cta;
+    const int n_groups = (a.B + seqs_per_cta - 1) / seqs_per_cta;
+    const int n_iter = (n_groups - (int)blockIdx.x + (int)gridDim.x - 1) / (int)gridDim.x;  // same for the whole CTA
+
+    auto seq_of = [&](int i) -> int {
+        const int b = ((int)blockIdx.x + i * (int)gridDim.x) * seqs_per_cta + sic;
+        return (lane_used && i < n_iter && b < a.B) ? b : -1;
+    };
+    auto load_len = [&](int b) -> int {
+        if (b < 0) return 0;
+        const bool rst = a.reset_mask ? (a.reset_mask[b] != 0) : (a.reset_first != 0);
+        return rst ? 0 : a.len[b];
+    };
+    auto slot_addr = [&](int stage, int slot) -> uint32_t {
+        return (uint32_t)__cvta_generic_to_shared(slots_mem + ((size_t)stage * n_slots + slot) * kTokThreads + tid);
+    };
+    // rows of the cache this thread must fetch for a sequence whose length (before the step) is len
+    auto rows_to_read = [&](int len) -> int { return (len < 0 || len + 1 > a.cap) ? 0 : len; };
+    auto issue = [&](int i, int len) {
+        const int b = seq_of(i);
+        if (b >= 0) {
+            const int stage = i % kStages;
+            const size_t slab = (size_t)b * a.H + h;
+            cp_async16(slot_addr(stage, 0), reinterpret_cast<const bf16*>(a.q) + slab * HD + sub * 8);
+            cp_async16(slot_addr(stage, 1), reinterpret_cast<const bf16*>(a.k_new) + slab * HD + sub * 8);
+            cp_async16(slot_addr(stage, 2), reinterpret_cast<const bf16*>(a.v_new) + slab * HD + sub * 8);
+            const bf16* cache = reinterpret_cast<const bf16*>(a.kv) + slab * a.cap * 2 * HD + sub * 8;
+            const int n = rows_to_read(len);
+            for (int r = 0; r < n; ++r) {
+                cp_async16(slot_addr(stage, 3 + 2 * r), cache + (size_t)r * 2 * HD);
+                cp_async16(slot_addr(stage, 4 + 2 * r), cache + (size_t)r * 2 * HD + HD);
+            }
+        }
+    };
+
+    // lens[d] = length of the sequence of group (i + d).  A length is needed when the copies of
+    // its group are issued (kDepth groups ahead) and is itself a DRAM read, so it is requested
+    // kLenAhead groups before that.
+    constexpr int kLenAhead = 3, kLens = kDepth + kLenAhead;
+    int lens[kLens];
+#pragma unroll
+    for (int d = 0; d < kLens; ++d) lens[d] = load_len(seq_of(d));
+#pragma unroll
+    for (int d = 0; d < kDepth; ++d) {
+        issue(d, lens[d]);
+        cp_async_commit();
+    }
+
+    for (int i = 0; i < n_iter; ++i) {
+        const int len_ahead = load_len(seq_of(i + kLens));
+        issue(i + kDepth, lens[kDepth]);
+        cp_async_commit();
+        cp_async_wait<kDepth>();  // the copies of group i have landed
+
+        const int b = seq_of(i);
+        const int len_raw = lens[0];
+        const bool overflow = len_raw < 0 || len_raw + 1 > a.cap;
+        const int n_old = (b >= 0 && !overflow) ? len_raw : 0;
+        const int stage = i % kStages;
+        const uint4* my = slots_mem + (size_t)stage * n_slots * kTokThreads + tid;
+        uint4 qr = make_uint4(0, 0, 0, 0), kr = qr, vr = qr;
+        if (b >= 0) {
+            qr = my[0];
+            kr = my[kTokThreads];
+            vr = my[2 * kTokThreads];
+        }
+        float qf[8];
+        unpack8(qr, qf);
+#pragma unroll
+        for (int d = 0; d < 8; ++d) qf[d] *= a.scale_log2;
+        // all scores first (independent dot products and shuffles), then one max, the exponentials
+        // and the weighted sum: with at most kMaxRows + 1 rows nothing needs a running rescale
+        uint4 vc[kMaxRows];
+        float sc[kMaxRows + 1];
+#pragma unroll
+        for (int r = 0; r < kMaxRows; ++r) {
+            const bool v = r < n_old;
+            const uint4 kc = v ? my[(size_t)(3 + 2 * r) * kTokThreads] : make_uint4(0, 0, 0, 0);
+            vc[r] = v ? my[(size_t)(4 + 2 * r) * kTokThreads] : make_uint4(0, 0, 0, 0);
+            const float d = row_sum<LPR>(dot8(qf, kc));
+            sc[r] = v ? d : kNegInf;
+        }
+        {
+            const float d = row_sum<LPR>(dot8(qf, kr));
+            sc[kMaxRows] = (b >= 0 && !overflow) ? d : kNegInf;
+        }
+        float mx = sc[kMaxRows];
+#pragma unroll
+        for (int r = 0; r < kMaxRows; ++r) mx = fmaxf(mx, sc[r]);
+        float l = 0.f, acc[8] = {0.f, 0.f, 0.f, 0.f, 0.f, 0.f, 0.f, 0.f};
+        if (mx != kNegInf) {
+#pragma unroll
+            for (int r = 0; r < kMaxRows; ++r) {
+                const float pr = ex2(sc[r] - mx);  // 0 for masked rows
+                l += pr;
+                fma8(acc, pr, vc[r]);
+            }
+            const float pn = ex2(sc[kMaxRows] - mx);
+            l += pn;
+            fma8(acc, pn, vr);
+        }
+        if (b >= 0) {
+            const size_t slab = (size_t)b * a.H + h;
+            if (!overflow) {
+                bf16* cache = reinterpret_cast<bf16*>(a.kv) + slab * a.cap * 2 * HD + sub * 8;
+                *reinterpret_cast<uint4*>(cache + (size_t)len_raw * 2 * HD) = kr;
+                *reinterpret_cast<uint4*>(cache + (size_t)len_raw * 2 * HD + HD) = vr;
+            }
+            float o[8];
+            const float inv = l > 0.f ? 1.f / l : 0.f;
+#pragma unroll
+            for (int d = 0; d < 8; ++d) o[d] = acc[d] * inv;
+            *reinterpret_cast<uint4*>(reinterpret_cast<bf16*>(a.out) + slab * HD + sub * 8) = pack8(o);
+        }
+        __syncthreads();  // all heads hold this group's (and the prefetched groups') lengths in registers
+        if (b >= 0 && within == 0) {
+            if (overflow)
+                raise_status(a.dev_status, BT_DEV_OVERFLOW);
+            else
+                a.len[b] = len_raw + 1;
+        }
+#pragma unroll
+        for (int d = 0; d + 1 < kLens; ++d) lens[d] = lens[d + 1];
+        lens[kLens - 1] = len_ahead;
+    }
+    cp_async_wait<0>();
+}
+
+static int sm_count()
+{
+    static int n = 0;
+    if (n == 0) {
+        int dev = 0;
+        if (cudaGetDevice(&dev) != cudaSuccess || cudaDeviceGetAttribute(&n, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess || n <= 0)
+            n = 148;
+    }
+    return n;
+}
+
+#ifndef BT_TOK_DEPTH4
+#define BT_TOK_DEPTH4 1
+#endif
+#ifndef BT_TOK_CTAS4
+#define BT_TOK_CTAS4 2
+#endif
+
+template <int HD, int kDepth, int kMaxRows, int kCtasPerSm>
+static cudaError_t launch_pipelined(const TokenArgs& a, int spc, int tps, cudaStream_t stream)
+{
+    constexpr size_t smem = (size_t)(kDepth + 1) * (3 + 2 * kMaxRows) * kTokThreads * sizeof(uint4);
+    static_assert(smem * kCtasPerSm <= 224 * 1024, "slots do not fit in shared memory");
+    static bool attr_set = false;
+    if (!attr_set) {
+        cudaError_t e = cudaFuncSetAttribute(token_step_pipelined_kernel<HD, kDepth, kMaxRows, kCtasPerSm>,
+                                             cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+        if (e != cudaSuccess) return e;
+        attr_set = true;
+    }
+    const int n_groups = (a.B + spc - 1) / spc;
+    const int slots = sm_count() * kCtasPerSm;
+    const int grid = n_groups < slots ? n_groups : slots;
+    token_step_pipelined_kernel<HD, kDepth, kMaxRows, kCtasPerSm><<<grid, kTokThreads, smem, stream>>>(a, spc, tps);
+    return cudaGetLastError();
+}
+
 cudaError_t launch_token_decode(const TokenArgs& a, cudaStream_t stream)
 {
     const int lpr = a.hd / 8;
     const int tps = a.H * lpr;  // threads per sequence (validated <= 256 by the caller)
-    int spc = 256 / tps;
+    if (a.n_q == 1 && a.k_new != nullptr && a.cap - 1 <= 8) {
+        // hot path: persistent pipelined kernel; deeper pipeline when the slots are small
+        int spc_p = kTokThreads / tps;
+        if (spc_p > a.B) spc_p = a.B;
+        if (a.cap - 1 <= 4)
+            return a.hd == 64 ? launch_pipelined<64, BT_TOK_DEPTH4, 4, BT_TOK_CTAS4>(a, spc_p, tps, stream)
+                              : launch_pipelined<128, BT_TOK_DEPTH4, 4, BT_TOK_CTAS4>(a, spc_p, tps, stream);
+        return a.hd == 64 ? launch_pipelined<64, 1, 8, 1>(a, spc_p, tps, stream)
+                          : launch_pipelined<128, 1, 8, 1>(a, spc_p, tps, stream);
+    }
+    int spc = BT_TOK_THREADS / tps;
     if (spc < 1) spc = 1;
     if (spc > a.B) spc = a.B;
     const int threads = ((spc * tps + 31) / 32) * 32;
