@@ -31,7 +31,12 @@ FALLBACK_PEAKS = {"hbm_gbs": 6650.0, "bf16_tflops": 1590.0, "bf16_tflops_sustain
 
 # DRAM traffic per launch of the dominant kernel, from the ncu captures summarised under profiles/
 # (dram__bytes_read.sum + dram__bytes_write.sum); None until a capture exists.
-NCU_TRAFFIC_BYTES = {"block_decode": None, "token_decode": None, "block_prefill": None}
+NCU_TRAFFIC_BYTES = {
+    # profiles/block_decode_kernel_config2.md: 272.6 MB on the B=128 capture, traffic is proportional to B
+    "block_decode": 545.2e6,
+    "token_decode": None,
+    "block_prefill": None,
+}
 
 
 def peaks():
