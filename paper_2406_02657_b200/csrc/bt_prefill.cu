@@ -2,15 +2,16 @@
 // the prefill stage processes all prompt blocks in parallel; causal over blocks).
 //
 // One CTA owns 128 query blocks of one (sequence, head) and walks the key/value blocks
-// 0 .. diagonal in tiles of 128:
-//   warp 4 (one lane): TMA producer - Q once, then K and V tiles into a 2-stage ring
-//   warp 5 (one lane): tcgen05.mma issuer - S = Q K^T into a double-buffered TMEM accumulator,
-//                      O += P V into a second TMEM accumulator
+// 0 .. diagonal in tiles of 128; two CTAs share an SM (96 KB of shared memory and 256 tensor-
+// memory columns each), so one CTA's softmax overlaps the other's MMAs and loads:
+//   warp 4 (one lane): TMA producer - Q once, then K and V tiles (K_j+1 lands while tile j is in
+//                      its softmax, V_j+1 while tile j+1 computes its scores)
+//   warp 5 (one lane): tcgen05.mma issuer - S = Q K^T into tensor memory, then O += P V with P read
+//                      from tensor memory (the probabilities never visit shared memory)
 //   warps 0-3        : softmax - each thread owns one query row (= one TMEM lane): row maximum,
-//                      exp2, bf16 P written to shared memory in the 128-byte-swizzled K-major
-//                      layout the MMA reads, running row sum; O is rescaled in TMEM only when the
-//                      row maximum grew by more than 2^8 (otherwise the old reference is kept,
-//                      which is exact because O and the row sum share the reference)
+//                      exp2, bf16 P written in place over the S columns, running row sum; O is
+//                      rescaled in TMEM only when the row maximum grew by more than 2^8 (otherwise
+//                      the old reference is kept, exact because O and the row sum share it)
 // All waits are bounded: a wait that runs out raises BT_DEV_TIMEOUT and the CTA winds down.
 #include <cuda.h>
 
@@ -28,7 +29,7 @@ constexpr uint32_t kSpinLimit = 1u << 22;
 constexpr float kRescaleThreshold = 8.0f;  // log2 units
 
 // ---- barrier slots in shared memory
-enum { B_QFULL = 0, B_KFULL = 1, B_VFULL = 3, B_KVEMPTY = 5, B_SFULL = 7, B_SEMPTY = 9, B_PFULL = 11, B_PVDONE = 12, B_COUNT = 13 };
+enum { B_QFULL = 0, B_KFULL, B_VFULL, B_KEMPTY, B_VEMPTY, B_SFULL, B_PFULL, B_OFULL, B_COUNT };
 
 __device__ __forceinline__ uint32_t smem_u32(const void* p) { return (uint32_t)__cvta_generic_to_shared(p); }
 
@@ -155,15 +156,39 @@ struct Params {
     float scale_log2;
 };
 
-template <int HD>
-constexpr int smem_bytes()
+// 16 consecutive 32-bit columns of this thread's TMEM lane (32 packed bf16).
+__device__ __forceinline__ void tmem_st16(uint32_t taddr, const uint32_t (&v)[16])
 {
-    // Q + 2 K stages + 2 V stages (HD/64 boxes each) + P (2 boxes) + barriers, plus 1024 to align
-    return 1024 + (HD / 64) * kBoxBytes * 5 + 2 * kBoxBytes + 256;
+    asm volatile(
+        "tcgen05.st.sync.aligned.32x32b.x16.b32 [%0], "
+        "{%1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15, %16};"
+        ::"r"(taddr), "r"(v[0]), "r"(v[1]), "r"(v[2]), "r"(v[3]), "r"(v[4]), "r"(v[5]), "r"(v[6]), "r"(v[7]),
+          "r"(v[8]), "r"(v[9]), "r"(v[10]), "r"(v[11]), "r"(v[12]), "r"(v[13]), "r"(v[14]), "r"(v[15])
+        : "memory");
+}
+
+// D[tmem] (+)= A[tmem] * B[smem]: A (the bf16 probabilities) is read from tensor memory.
+__device__ __forceinline__ void mma_bf16_ts(uint32_t tmem_d, uint32_t tmem_a, uint64_t bdesc, uint32_t idesc, uint32_t accumulate)
+{
+    asm volatile(
+        "{\n\t.reg .pred p;\n\t"
+        "setp.ne.b32 p, %4, 0;\n\t"
+        "tcgen05.mma.cta_group::1.kind::f16 [%0], [%1], %2, %3, p;\n\t}"
+        ::"r"(tmem_d), "r"(tmem_a), "l"(bdesc), "r"(idesc), "r"(accumulate)
+        : "memory");
 }
 
 template <int HD>
-__global__ void __launch_bounds__(kThreads, 1)
+constexpr int smem_bytes()
+{
+    // Q, K, V tiles (HD/64 boxes each) + barriers, plus 1024 to align
+    return 1024 + (HD / 64) * kBoxBytes * 3 + 256;
+}
+
+constexpr uint32_t kTmemCols = 256;  // S/P: 128 columns, O: up to 128 columns; two CTAs fit in the SM's 512
+
+template <int HD>
+__global__ void __launch_bounds__(kThreads, 2)
 block_prefill_tc_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_constant__ CUtensorMap mapK,
                         const __grid_constant__ CUtensorMap mapV, Params p)
 {
@@ -171,16 +196,15 @@ block_prefill_tc_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_c
     constexpr uint32_t TILE_BYTES = NB * kBoxBytes;
     constexpr uint32_t IDESC_S = make_idesc(BM, BN, false);
     constexpr uint32_t IDESC_O = make_idesc(BM, HD, true);
-    constexpr uint32_t COL_S = 0, COL_O = 2 * BN;  // TMEM columns: S0 | S1 | O
+    constexpr uint32_t COL_S = 0, COL_O = BN;   // TMEM columns: S (fp32) / P (bf16 pairs, in place) | O
 
     extern __shared__ uint8_t smem_raw[];
     const uint32_t base = (smem_u32(smem_raw) + 1023u) & ~1023u;
     uint8_t* gen_base = smem_raw + (base - smem_u32(smem_raw));
     const uint32_t sQ = base;
-    const uint32_t sK = sQ + TILE_BYTES;       // [2][TILE_BYTES]
-    const uint32_t sV = sK + 2 * TILE_BYTES;   // [2][TILE_BYTES]
-    const uint32_t sP = sV + 2 * TILE_BYTES;   // [2 boxes]
-    const uint32_t sBar = sP + 2 * kBoxBytes;  // B_COUNT x 8 bytes
+    const uint32_t sK = sQ + TILE_BYTES;
+    const uint32_t sV = sK + TILE_BYTES;
+    const uint32_t sBar = sV + TILE_BYTES;      // B_COUNT x 8 bytes
     uint8_t* gen_tail = gen_base + (sBar - base);
     uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(gen_tail + B_COUNT * 8);
     volatile int* abort_flag = reinterpret_cast<volatile int*>(gen_tail + B_COUNT * 8 + 8);
@@ -193,20 +217,18 @@ block_prefill_tc_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_c
 
     if (threadIdx.x == 0) {
         mbar_init(bar(B_QFULL), 1);
-        for (int s = 0; s < 2; ++s) {
-            mbar_init(bar(B_KFULL + s), 1);
-            mbar_init(bar(B_VFULL + s), 1);
-            mbar_init(bar(B_KVEMPTY + s), 1);
-            mbar_init(bar(B_SFULL + s), 1);
-            mbar_init(bar(B_SEMPTY + s), 128);
-        }
+        mbar_init(bar(B_KFULL), 1);
+        mbar_init(bar(B_VFULL), 1);
+        mbar_init(bar(B_KEMPTY), 1);
+        mbar_init(bar(B_VEMPTY), 1);
+        mbar_init(bar(B_SFULL), 1);
         mbar_init(bar(B_PFULL), 128);
-        mbar_init(bar(B_PVDONE), 1);
+        mbar_init(bar(B_OFULL), 1);
         *abort_flag = 0;
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     }
-    if (warp == 0) {  // allocate all 512 TMEM columns (S0, S1, O); this warp also frees them
-        asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(tmem_slot)), "r"(512u) : "memory");
+    if (warp == 0) {  // this warp allocates the CTA's tensor-memory columns and frees them at the end
+        asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(tmem_slot)), "r"(kTmemCols) : "memory");
         asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
     }
     tc_fence_before();
@@ -223,54 +245,46 @@ block_prefill_tc_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_c
             mbar_expect_tx(bar(B_QFULL), TILE_BYTES);
             for (int bx = 0; bx < NB; ++bx) tma_load_3d(sQ + bx * kBoxBytes, &mapQ, bar(B_QFULL), bx * 64, qt * BM, bh);
             for (int j = 0; j < n_kv; ++j) {
-                const int st = j & 1;
-                if (j >= 2 && !mbar_wait(bar(B_KVEMPTY + st), ((j >> 1) - 1) & 1, abort_flag, p.dev_status)) break;
-                mbar_expect_tx(bar(B_KFULL + st), TILE_BYTES);
-                for (int bx = 0; bx < NB; ++bx)
-                    tma_load_3d(sK + st * TILE_BYTES + bx * kBoxBytes, &mapK, bar(B_KFULL + st), bx * 64, j * BN, bh);
-                mbar_expect_tx(bar(B_VFULL + st), TILE_BYTES);
-                for (int bx = 0; bx < NB; ++bx)
-                    tma_load_3d(sV + st * TILE_BYTES + bx * kBoxBytes, &mapV, bar(B_VFULL + st), bx * 64, j * BN, bh);
+                // K_j may land once S_{j-1} has consumed K_{j-1}; V_j once P_{j-1} V_{j-1} has consumed V_{j-1}
+                if (j >= 1 && !mbar_wait(bar(B_KEMPTY), (j - 1) & 1, abort_flag, p.dev_status)) break;
+                mbar_expect_tx(bar(B_KFULL), TILE_BYTES);
+                for (int bx = 0; bx < NB; ++bx) tma_load_3d(sK + bx * kBoxBytes, &mapK, bar(B_KFULL), bx * 64, j * BN, bh);
+                if (j >= 1 && !mbar_wait(bar(B_VEMPTY), (j - 1) & 1, abort_flag, p.dev_status)) break;
+                mbar_expect_tx(bar(B_VFULL), TILE_BYTES);
+                for (int bx = 0; bx < NB; ++bx) tma_load_3d(sV + bx * kBoxBytes, &mapV, bar(B_VFULL), bx * 64, j * BN, bh);
             }
         }
     } else if (warp == 5) {
         // ------------------------------------------------------------------ MMA issuer
         if (lane == 0) {
             bool ok = mbar_wait(bar(B_QFULL), 0, abort_flag, p.dev_status);
-            auto issue_pv = [&](int t) -> bool {
-                const int st = t & 1;
-                if (!mbar_wait(bar(B_PFULL), t & 1, abort_flag, p.dev_status)) return false;
-                if (!mbar_wait(bar(B_VFULL + st), (t >> 1) & 1, abort_flag, p.dev_status)) return false;
-                tc_fence_after();
-#pragma unroll
-                for (int kk = 0; kk < BN / 16; ++kk) {
-                    // A = P, K-major: 16 kv columns = 32 bytes inside the swizzled 128-byte row
-                    const uint64_t a = make_desc(sP + (kk >> 2) * kBoxBytes + (kk & 3) * 32, 16, 1024);
-                    // B = V, MN-major: 16 kv rows = 2048 bytes; next 64 head dims one box further
-                    const uint64_t b = make_desc(sV + st * TILE_BYTES + kk * 2048, kBoxBytes, 1024);
-                    mma_bf16(tmem + COL_O, a, b, IDESC_O, (t > 0 || kk > 0) ? 1u : 0u);
-                }
-                mma_commit(bar(B_KVEMPTY + st));
-                mma_commit(bar(B_PVDONE));
-                return true;
-            };
             for (int j = 0; ok && j < n_kv; ++j) {
-                const int st = j & 1;
-                ok = mbar_wait(bar(B_KFULL + st), (j >> 1) & 1, abort_flag, p.dev_status);
-                if (ok && j >= 2) ok = mbar_wait(bar(B_SEMPTY + st), ((j >> 1) - 1) & 1, abort_flag, p.dev_status);
+                ok = mbar_wait(bar(B_KFULL), j & 1, abort_flag, p.dev_status);
                 if (!ok) break;
                 tc_fence_after();
+                // S_j overwrites the columns P_{j-1} lived in: MMAs of one thread execute in issue
+                // order, and P_{j-1} V_{j-1} was issued before this.
 #pragma unroll
                 for (int kk = 0; kk < HD / 16; ++kk) {
                     const uint32_t off = (kk >> 2) * kBoxBytes + (kk & 3) * 32;
-                    const uint64_t a = make_desc(sQ + off, 16, 1024);
-                    const uint64_t b = make_desc(sK + st * TILE_BYTES + off, 16, 1024);
-                    mma_bf16(tmem + COL_S + st * BN, a, b, IDESC_S, kk > 0 ? 1u : 0u);
+                    mma_bf16(tmem + COL_S, make_desc(sQ + off, 16, 1024), make_desc(sK + off, 16, 1024), IDESC_S, kk > 0 ? 1u : 0u);
                 }
-                mma_commit(bar(B_SFULL + st));
-                if (j >= 1) ok = issue_pv(j - 1);
+                mma_commit(bar(B_SFULL));
+                mma_commit(bar(B_KEMPTY));
+                ok = mbar_wait(bar(B_PFULL), j & 1, abort_flag, p.dev_status) &&
+                     mbar_wait(bar(B_VFULL), j & 1, abort_flag, p.dev_status);
+                if (!ok) break;
+                tc_fence_after();
+#pragma unroll
+                for (int kk = 0; kk < BN / 16; ++kk) {
+                    // A = P from tensor memory: 16 kv columns = 8 packed 32-bit columns;
+                    // B = V, MN-major: 16 kv rows = 2048 bytes; next 64 head dims one box further
+                    mma_bf16_ts(tmem + COL_O, tmem + COL_S + kk * 8, make_desc(sV + kk * 2048, kBoxBytes, 1024), IDESC_O,
+                                (j > 0 || kk > 0) ? 1u : 0u);
+                }
+                mma_commit(bar(B_VEMPTY));
+                if (j == n_kv - 1) mma_commit(bar(B_OFULL));
             }
-            if (ok) issue_pv(n_kv - 1);
         }
     } else {
         // ------------------------------------------------------------------ softmax: thread = query row
@@ -280,12 +294,11 @@ block_prefill_tc_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_c
         float m_ref = kNegInf, l = 0.f;
         bool ok = true;
         for (int j = 0; j < n_kv; ++j) {
-            const int st = j & 1;
             const bool diag = (j == qt);
-            ok = mbar_wait(bar(B_SFULL + st), (j >> 1) & 1, abort_flag, p.dev_status);
+            ok = mbar_wait(bar(B_SFULL), j & 1, abort_flag, p.dev_status);  // S_j ready; O settled (all earlier MMAs done)
             if (!ok) break;
             tc_fence_after();
-            const uint32_t s_addr = lane_base + COL_S + st * BN;
+            const uint32_t s_addr = lane_base + COL_S;
             // pass 1: row maximum over the allowed columns
             float mx = kNegInf;
 #pragma unroll 1
@@ -304,9 +317,6 @@ block_prefill_tc_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_c
                 m_ref = mx;
             }
             if (j > 0) {
-                ok = mbar_wait(bar(B_PVDONE), (j - 1) & 1, abort_flag, p.dev_status);  // P buffer free, O settled
-                if (!ok) break;
-                tc_fence_after();
                 if (__any_sync(0xffffffffu, grow_ref)) {
 #pragma unroll 1
                     for (int c0 = 0; c0 < HD; c0 += 32) {
@@ -316,11 +326,12 @@ block_prefill_tc_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_c
                         for (int i = 0; i < 32; ++i) o[i] *= factor;
                         tmem_st32(lane_base + COL_O + c0, o);
                     }
-                    tmem_wait_st();
                 }
                 l *= factor;
             }
-            // pass 2: P = 2^(s*scale - m_ref), bf16, into the swizzled K-major tile; row sum of what the MMA will see
+            // pass 2: P = 2^(s*scale - m_ref) as bf16 pairs, written in place over the S columns already
+            // consumed (chunk c of P lands in columns 16c..16c+15, inside S columns 0..32c+31); the row sum
+            // is taken over the rounded values the MMA will see
 #pragma unroll 1
             for (int c0 = 0; c0 < BN; c0 += 32) {
                 float v[32];
@@ -335,21 +346,13 @@ block_prefill_tc_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_c
                     packed[i >> 1] = w;
                     l += bf_lo(w) + bf_hi(w);
                 }
-                const uint32_t box = sP + (c0 >> 6) * kBoxBytes + row * 128;
-#pragma unroll
-                for (int q4 = 0; q4 < 4; ++q4) {
-                    const uint32_t chunk = (uint32_t)(((c0 & 63) >> 3) + q4) ^ (uint32_t)(row & 7);
-                    asm volatile("st.shared.v4.u32 [%0], {%1, %2, %3, %4};" ::"r"(box + chunk * 16), "r"(packed[4 * q4]),
-                                 "r"(packed[4 * q4 + 1]), "r"(packed[4 * q4 + 2]), "r"(packed[4 * q4 + 3])
-                                 : "memory");
-                }
+                tmem_st16(s_addr + (c0 >> 1), packed);
             }
+            tmem_wait_st();
             tc_fence_before();
-            asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
-            mbar_arrive(bar(B_SEMPTY + st));
             mbar_arrive(bar(B_PFULL));
         }
-        if (ok) ok = mbar_wait(bar(B_PVDONE), (n_kv - 1) & 1, abort_flag, p.dev_status);
+        if (ok) ok = mbar_wait(bar(B_OFULL), 0, abort_flag, p.dev_status);
         if (ok) {
             tc_fence_after();
             const float inv = l > 0.f ? 1.f / l : 0.f;
@@ -375,7 +378,7 @@ block_prefill_tc_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_c
     __syncthreads();
     if (warp == 0) {
         tc_fence_after();
-        asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem), "r"(512u) : "memory");
+        asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem), "r"(kTmemCols) : "memory");
     }
 }
 
