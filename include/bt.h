@@ -122,6 +122,31 @@ bt_status bt_block_decode_attn(const bt_config* cfg, const bt_block_cache* cache
                                uint32_t* dev_status, void* stream);
 
 /*
+ * bt_block_decode_attn for callers that cannot supply a workspace.  (The paper has no
+ * counterpart: this is a property of the library, not of the method.)  It computes exactly what
+ * bt_block_decode_attn computes, with the per-split partials kept in a fixed array inside the
+ * loaded library instead of caller memory.  It is meant for hosts that have no device memory
+ * left to give (a serving process whose pool took the whole GPU at start-up) or that must not
+ * allocate where they call from (cudaMalloc synchronises the whole device, which a decode loop
+ * with a latency budget cannot accept).  Neither this call nor anything it reaches allocates or
+ * frees device memory.
+ *   - Limit: bt_workspace_bytes(cfg) must not exceed BT_STATIC_WORKSPACE_BYTES, else
+ *     BT_ERR_WORKSPACE is returned and nothing is launched.  Every GPU on which the library is
+ *     loaded holds that many bytes until the process exits.
+ *   - The first call on each device whose config splits the row range looks up the array's
+ *     address on that device (the device must be current, as for every call here, and own the
+ *     buffers passed in).  Make that first call outside any stream capture.
+ *   - All calls on one device share the array.  It needs no clearing (every partial is written
+ *     before it is read within one call, so what an earlier call left behind is never seen), but
+ *     two calls that can overlap on the GPU (different streams, no dependency) race on it:
+ *     order them, or give one of them bt_block_decode_attn with its own workspace.
+ * Other arguments, results and errors are those of bt_block_decode_attn.
+ */
+#define BT_STATIC_WORKSPACE_BYTES (2u << 20) /* 2 MiB */
+bt_status bt_block_decode_attn_noalloc(const bt_config* cfg, const bt_block_cache* cache, int layer,
+                                       const void* q, void* out, uint32_t* dev_status, void* stream);
+
+/*
  * Block boundary of the token decoder (Figure 1; section 2.4): the local K,V of a finished
  * block are never read again, so the cache is dropped by zeroing its length; no data is
  * cleared.  seq_mask: NULL resets every sequence, else uint8 [B], non-zero = reset.

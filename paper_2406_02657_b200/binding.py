@@ -20,7 +20,7 @@ BT_DEV_OK, BT_DEV_OVERFLOW, BT_DEV_EMPTY, BT_DEV_TIMEOUT = 0, 1, 2, 4
 EXPORTS = [
     "bt_version", "bt_status_string", "bt_decode_splits", "bt_workspace_bytes", "bt_block_kv_append",
     "bt_block_decode_attn", "bt_local_kv_reset", "bt_local_kv_append", "bt_token_decode_attn",
-    "bt_block_prefill_attn", "bt_block_decode_step_host",
+    "bt_block_prefill_attn", "bt_block_decode_step_host", "bt_block_decode_attn_noalloc",
 ]
 
 
@@ -67,6 +67,7 @@ def _load() -> ctypes.CDLL:
     lib.bt_block_prefill_attn.argtypes = [cfgp, vp, vp, vp, i32, ctypes.c_int64, vp, vp, vp]
     lib.bt_block_decode_step_host.argtypes = [cfgp, ctypes.POINTER(bt_block_cache), i32, vp, vp, vp, vp,
                                               vp, vp, vp, vp, vp, u64, vp, vp]
+    lib.bt_block_decode_attn_noalloc.argtypes = [cfgp, ctypes.POINTER(bt_block_cache), i32, vp, vp, vp, vp]
     for name in EXPORTS[4:]:
         getattr(lib, name).restype = ctypes.c_int
     return lib
@@ -159,6 +160,17 @@ def bt_block_decode_attn(cfg, cache: BlockCache, layer, q, out, workspace=None, 
     _check(_lib.bt_block_decode_attn(ctypes.byref(cfg), ctypes.byref(cache.c), layer, _ptr(q), _ptr(out),
                                      _ptr(workspace), ws_bytes, _ptr(dev_status), _stream(stream)),
            "bt_block_decode_attn")
+
+
+BT_STATIC_WORKSPACE_BYTES = 2 << 20
+
+
+def bt_block_decode_attn_noalloc(cfg, cache: BlockCache, layer, q, out, dev_status=None, stream=None):
+    """bt_block_decode_attn with the split scratch inside the library (no workspace argument): for
+    callers that cannot allocate device memory.  Rejects configs whose scratch would exceed
+    BT_STATIC_WORKSPACE_BYTES; calls on one device share the scratch, so do not overlap them."""
+    _check(_lib.bt_block_decode_attn_noalloc(ctypes.byref(cfg), ctypes.byref(cache.c), layer, _ptr(q), _ptr(out),
+                                             _ptr(dev_status), _stream(stream)), "bt_block_decode_attn_noalloc")
 
 
 def bt_local_kv_reset(cfg, cache: LocalCache, layer, seq_mask=None, stream=None):
