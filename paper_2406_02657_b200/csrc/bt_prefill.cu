@@ -4,14 +4,17 @@
 // One CTA owns 128 query blocks of one (sequence, head) and walks the key/value blocks
 // 0 .. diagonal in tiles of 128; two CTAs share an SM (96 KB of shared memory and 256 tensor-
 // memory columns each), so one CTA's softmax overlaps the other's MMAs and loads:
-//   warp 4 (one lane): TMA producer - Q once, then K and V tiles (K_j+1 lands while tile j is in
-//                      its softmax, V_j+1 while tile j+1 computes its scores)
-//   warp 5 (one lane): tcgen05.mma issuer - S = Q K^T into tensor memory, then O += P V with P read
-//                      from tensor memory (the probabilities never visit shared memory)
-//   warps 0-3        : softmax - each thread owns one query row (= one TMEM lane): row maximum,
-//                      exp2, bf16 P written in place over the S columns, running row sum; O is
-//                      rescaled in TMEM only when the row maximum grew by more than 2^8 (otherwise
-//                      the old reference is kept, exact because O and the row sum share it)
+//   warp 4 (one lane): TMA producer and tcgen05.mma issuer - Q once, then per tile S = Q K^T into
+//                      tensor memory and O += P V with P read from tensor memory (the probabilities
+//                      never visit shared memory); K_j+1 is requested as soon as S_j has consumed
+//                      K_j, V_j+1 as soon as P_j V_j has consumed V_j
+//   warps 0-3        : softmax - each thread owns one query row (= one TMEM lane) and holds its
+//                      128 scores in registers: one batch of tensor-memory loads, row maximum,
+//                      exp2 (packed fp32x2 multiply-adds around it), bf16 P written over the S
+//                      columns, running row sum; on the diagonal tile a warp skips the column
+//                      chunks that are masked for all of its rows.  O is rescaled in TMEM only when
+//                      the row maximum grew by more than 2^8 (otherwise the old reference is kept,
+//                      exact because O and the row sum share it)
 // All waits are bounded: a wait that runs out raises BT_DEV_TIMEOUT and the CTA winds down.
 #include <cuda.h>
 
@@ -24,7 +27,7 @@ namespace pf {
 constexpr int BM = 128;             // query rows per CTA
 constexpr int BN = 128;             // key/value rows per tile
 constexpr int kBoxBytes = 128 * 128;  // one TMA box: 128 rows x 64 bf16 (128 bytes, swizzled)
-constexpr int kThreads = 192;
+constexpr int kThreads = 160;
 constexpr uint32_t kSpinLimit = 1u << 22;
 constexpr float kRescaleThreshold = 8.0f;  // log2 units
 
@@ -178,6 +181,72 @@ __device__ __forceinline__ void mma_bf16_ts(uint32_t tmem_d, uint32_t tmem_a, ui
         : "memory");
 }
 
+// Issue (without waiting) the load of 32 consecutive 32-bit columns of this thread's TMEM lane
+// into r[0..31].  The registers hold the data only after tmem_ld_fence32 on the same registers.
+__device__ __forceinline__ void tmem_ld32_issue(uint32_t taddr, uint32_t* r)
+{
+    asm volatile(
+        "tcgen05.ld.sync.aligned.32x32b.x32.b32 "
+        "{%0, %1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15, "
+        "%16, %17, %18, %19, %20, %21, %22, %23, %24, %25, %26, %27, %28, %29, %30, %31}, [%32];"
+        : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]), "=r"(r[4]), "=r"(r[5]), "=r"(r[6]), "=r"(r[7]),
+          "=r"(r[8]), "=r"(r[9]), "=r"(r[10]), "=r"(r[11]), "=r"(r[12]), "=r"(r[13]), "=r"(r[14]), "=r"(r[15]),
+          "=r"(r[16]), "=r"(r[17]), "=r"(r[18]), "=r"(r[19]), "=r"(r[20]), "=r"(r[21]), "=r"(r[22]), "=r"(r[23]),
+          "=r"(r[24]), "=r"(r[25]), "=r"(r[26]), "=r"(r[27]), "=r"(r[28]), "=r"(r[29]), "=r"(r[30]), "=r"(r[31])
+        : "r"(taddr)
+        : "memory");
+}
+// Placed after tmem_wait_ld(): makes every later use of r[0..31] depend on a statement that follows
+// the wait, so no consumer can be scheduled ahead of it.  Emits no instruction.
+__device__ __forceinline__ void tmem_ld_fence32(uint32_t* r)
+{
+    asm volatile(""
+        : "+r"(r[0]), "+r"(r[1]), "+r"(r[2]), "+r"(r[3]), "+r"(r[4]), "+r"(r[5]), "+r"(r[6]), "+r"(r[7]),
+          "+r"(r[8]), "+r"(r[9]), "+r"(r[10]), "+r"(r[11]), "+r"(r[12]), "+r"(r[13]), "+r"(r[14]), "+r"(r[15]),
+          "+r"(r[16]), "+r"(r[17]), "+r"(r[18]), "+r"(r[19]), "+r"(r[20]), "+r"(r[21]), "+r"(r[22]), "+r"(r[23]),
+          "+r"(r[24]), "+r"(r[25]), "+r"(r[26]), "+r"(r[27]), "+r"(r[28]), "+r"(r[29]), "+r"(r[30]), "+r"(r[31])
+        :: "memory");
+}
+__device__ __forceinline__ void tmem_st16p(uint32_t taddr, const uint32_t* v)
+{
+    asm volatile(
+        "tcgen05.st.sync.aligned.32x32b.x16.b32 [%0], "
+        "{%1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15, %16};"
+        ::"r"(taddr), "r"(v[0]), "r"(v[1]), "r"(v[2]), "r"(v[3]), "r"(v[4]), "r"(v[5]), "r"(v[6]), "r"(v[7]),
+          "r"(v[8]), "r"(v[9]), "r"(v[10]), "r"(v[11]), "r"(v[12]), "r"(v[13]), "r"(v[14]), "r"(v[15])
+        : "memory");
+}
+
+// Packed fp32 pairs (one issue slot for two lanes' worth of work on sm_100).
+__device__ __forceinline__ uint64_t pack2(float lo, float hi)
+{
+    uint64_t d;
+    asm("mov.b64 %0, {%1, %2};" : "=l"(d) : "f"(lo), "f"(hi));
+    return d;
+}
+__device__ __forceinline__ void unpack2(uint64_t v, float& lo, float& hi)
+{
+    asm("mov.b64 {%0, %1}, %2;" : "=f"(lo), "=f"(hi) : "l"(v));
+}
+__device__ __forceinline__ uint64_t ffma2(uint64_t a, uint64_t b, uint64_t c)
+{
+    uint64_t d;
+    asm("fma.rn.f32x2 %0, %1, %2, %3;" : "=l"(d) : "l"(a), "l"(b), "l"(c));
+    return d;
+}
+__device__ __forceinline__ uint64_t fadd2(uint64_t a, uint64_t b)
+{
+    uint64_t d;
+    asm("add.rn.f32x2 %0, %1, %2;" : "=l"(d) : "l"(a), "l"(b));
+    return d;
+}
+__device__ __forceinline__ float fmax3(float a, float b, float c)
+{
+    float d;
+    asm("max.f32 %0, %1, %2, %3;" : "=f"(d) : "f"(a), "f"(b), "f"(c));
+    return d;
+}
+
 template <int HD>
 constexpr int smem_bytes()
 {
@@ -237,33 +306,22 @@ block_prefill_tc_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_c
     const uint32_t tmem = *tmem_slot;
 
     if (warp == 4) {
-        // ------------------------------------------------------------------ TMA producer
+        // ------------------------------------------------------------------ TMA producer + MMA issuer
         if (lane == 0) {
             asm volatile("prefetch.tensormap [%0];" ::"l"(&mapQ) : "memory");
             asm volatile("prefetch.tensormap [%0];" ::"l"(&mapK) : "memory");
             asm volatile("prefetch.tensormap [%0];" ::"l"(&mapV) : "memory");
-            mbar_expect_tx(bar(B_QFULL), TILE_BYTES);
-            for (int bx = 0; bx < NB; ++bx) tma_load_3d(sQ + bx * kBoxBytes, &mapQ, bar(B_QFULL), bx * 64, qt * BM, bh);
-            for (int j = 0; j < n_kv; ++j) {
-                // K_j may land once S_{j-1} has consumed K_{j-1}; V_j once P_{j-1} V_{j-1} has consumed V_{j-1}
-                if (j >= 1 && !mbar_wait(bar(B_KEMPTY), (j - 1) & 1, abort_flag, p.dev_status)) break;
+            auto load_k = [&](int j) {
                 mbar_expect_tx(bar(B_KFULL), TILE_BYTES);
                 for (int bx = 0; bx < NB; ++bx) tma_load_3d(sK + bx * kBoxBytes, &mapK, bar(B_KFULL), bx * 64, j * BN, bh);
-                if (j >= 1 && !mbar_wait(bar(B_VEMPTY), (j - 1) & 1, abort_flag, p.dev_status)) break;
+            };
+            auto load_v = [&](int j) {
                 mbar_expect_tx(bar(B_VFULL), TILE_BYTES);
                 for (int bx = 0; bx < NB; ++bx) tma_load_3d(sV + bx * kBoxBytes, &mapV, bar(B_VFULL), bx * 64, j * BN, bh);
-            }
-        }
-    } else if (warp == 5) {
-        // ------------------------------------------------------------------ MMA issuer
-        if (lane == 0) {
-            bool ok = mbar_wait(bar(B_QFULL), 0, abort_flag, p.dev_status);
-            for (int j = 0; ok && j < n_kv; ++j) {
-                ok = mbar_wait(bar(B_KFULL), j & 1, abort_flag, p.dev_status);
-                if (!ok) break;
-                tc_fence_after();
-                // S_j overwrites the columns P_{j-1} lived in: MMAs of one thread execute in issue
-                // order, and P_{j-1} V_{j-1} was issued before this.
+            };
+            // S_j = Q K_j^T.  It overwrites the columns P_{j-1} lived in: MMAs of one thread execute in
+            // issue order, and P_{j-1} V_{j-1} is always issued before S_j.
+            auto issue_s = [&]() {
 #pragma unroll
                 for (int kk = 0; kk < HD / 16; ++kk) {
                     const uint32_t off = (kk >> 2) * kBoxBytes + (kk & 3) * 32;
@@ -271,6 +329,24 @@ block_prefill_tc_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_c
                 }
                 mma_commit(bar(B_SFULL));
                 mma_commit(bar(B_KEMPTY));
+            };
+            mbar_expect_tx(bar(B_QFULL), TILE_BYTES);
+            for (int bx = 0; bx < NB; ++bx) tma_load_3d(sQ + bx * kBoxBytes, &mapQ, bar(B_QFULL), bx * 64, qt * BM, bh);
+            load_k(0);
+            load_v(0);
+            bool ok = mbar_wait(bar(B_QFULL), 0, abort_flag, p.dev_status) &&
+                      mbar_wait(bar(B_KFULL), 0, abort_flag, p.dev_status);
+            if (ok) {
+                tc_fence_after();
+                issue_s();
+            }
+            for (int j = 0; ok && j < n_kv; ++j) {
+                const bool more = j + 1 < n_kv;
+                if (more) {  // K_{j+1} may land once S_j has consumed K_j
+                    ok = mbar_wait(bar(B_KEMPTY), j & 1, abort_flag, p.dev_status);
+                    if (!ok) break;
+                    load_k(j + 1);
+                }
                 ok = mbar_wait(bar(B_PFULL), j & 1, abort_flag, p.dev_status) &&
                      mbar_wait(bar(B_VFULL), j & 1, abort_flag, p.dev_status);
                 if (!ok) break;
@@ -283,7 +359,19 @@ block_prefill_tc_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_c
                                 (j > 0 || kk > 0) ? 1u : 0u);
                 }
                 mma_commit(bar(B_VEMPTY));
-                if (j == n_kv - 1) mma_commit(bar(B_OFULL));
+                if (!more) {
+                    mma_commit(bar(B_OFULL));
+                    break;
+                }
+                // queue S_{j+1} behind P_j V_j so the tensor pipe never waits for this thread
+                ok = mbar_wait(bar(B_KFULL), (j + 1) & 1, abort_flag, p.dev_status);
+                if (!ok) break;
+                tc_fence_after();
+                issue_s();
+                // V_{j+1} may land once P_j V_j has consumed V_j
+                ok = mbar_wait(bar(B_VEMPTY), j & 1, abort_flag, p.dev_status);
+                if (!ok) break;
+                load_v(j + 1);
             }
         }
     } else {
@@ -299,16 +387,34 @@ block_prefill_tc_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_c
             if (!ok) break;
             tc_fence_after();
             const uint32_t s_addr = lane_base + COL_S;
-            // pass 1: row maximum over the allowed columns
-            float mx = kNegInf;
-#pragma unroll 1
-            for (int c0 = 0; c0 < BN; c0 += 32) {
-                float v[32];
-                tmem_ld32(s_addr + c0, v);
+            // On the diagonal tile the rows of warp w (32w .. 32w+31) see nothing right of column
+            // 32w+31: only column chunks 0..w are loaded and exponentiated, chunk w with a per-row mask.
+            const int nch = diag ? warp + 1 : BN / 32;
+            uint32_t sr[BN];
 #pragma unroll
-                for (int i = 0; i < 32; ++i)
-                    if (!diag || c0 + i <= row) mx = fmaxf(mx, v[i]);
+            for (int c = 0; c < BN / 32; ++c)
+                if (c < nch) tmem_ld32_issue(s_addr + c * 32, sr + c * 32);
+            tmem_wait_ld();
+#pragma unroll
+            for (int c = 0; c < BN / 32; ++c)
+                if (c < nch) tmem_ld_fence32(sr + c * 32);
+            if (diag) {  // masked scores become -inf: they drop out of the maximum and exponentiate to 0
+#pragma unroll
+                for (int c = 0; c < BN / 32; ++c)
+                    if (c == warp) {
+#pragma unroll
+                        for (int i = 0; i < 32; ++i)
+                            if (i > lane) sr[c * 32 + i] = __float_as_uint(kNegInf);
+                    }
             }
+            float mx = kNegInf;
+#pragma unroll
+            for (int c = 0; c < BN / 32; ++c)
+                if (c < nch) {
+#pragma unroll
+                    for (int i = 0; i < 32; i += 2)
+                        mx = fmax3(mx, __uint_as_float(sr[c * 32 + i]), __uint_as_float(sr[c * 32 + i + 1]));
+                }
             mx *= p.scale_log2;
             float factor = 1.f;
             const bool grow_ref = mx > m_ref + kRescaleThreshold;  // first tile: m_ref = -inf
@@ -329,24 +435,39 @@ block_prefill_tc_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_c
                 }
                 l *= factor;
             }
-            // pass 2: P = 2^(s*scale - m_ref) as bf16 pairs, written in place over the S columns already
-            // consumed (chunk c of P lands in columns 16c..16c+15, inside S columns 0..32c+31); the row sum
-            // is taken over the rounded values the MMA will see
-#pragma unroll 1
-            for (int c0 = 0; c0 < BN; c0 += 32) {
-                float v[32];
-                tmem_ld32(s_addr + c0, v);
-                uint32_t packed[16];
+            // P = 2^(s*scale - m_ref) as bf16 pairs over the S columns (chunk c of P lands in columns
+            // 16c .. 16c+15; every S column is already in registers).  The row sum is taken in fp32
+            // before the rounding: the rounding errors of the 128 terms average out in the normaliser.
+            const uint64_t sc2 = pack2(p.scale_log2, p.scale_log2), nm2 = pack2(-m_ref, -m_ref);
+            uint64_t l2a = pack2(0.f, 0.f), l2b = l2a;
 #pragma unroll
-                for (int i = 0; i < 32; i += 2) {
-                    float p0 = (!diag || c0 + i <= row) ? ex2(fmaf(v[i], p.scale_log2, -m_ref)) : 0.f;
-                    float p1 = (!diag || c0 + i + 1 <= row) ? ex2(fmaf(v[i + 1], p.scale_log2, -m_ref)) : 0.f;
-                    __nv_bfloat162 pk = __floats2bfloat162_rn(p0, p1);
-                    uint32_t w = *reinterpret_cast<uint32_t*>(&pk);
-                    packed[i >> 1] = w;
-                    l += bf_lo(w) + bf_hi(w);
+            for (int c = 0; c < BN / 32; ++c) {
+                uint32_t packed[16];
+                if (c < nch) {
+#pragma unroll
+                    for (int i = 0; i < 32; i += 4) {
+                        const uint32_t* e = sr + c * 32 + i;
+                        float x0, x1, x2, x3;
+                        unpack2(ffma2(pack2(__uint_as_float(e[0]), __uint_as_float(e[1])), sc2, nm2), x0, x1);
+                        unpack2(ffma2(pack2(__uint_as_float(e[2]), __uint_as_float(e[3])), sc2, nm2), x2, x3);
+                        const float p0 = ex2(x0), p1 = ex2(x1), p2 = ex2(x2), p3 = ex2(x3);
+                        l2a = fadd2(l2a, pack2(p0, p1));
+                        l2b = fadd2(l2b, pack2(p2, p3));
+                        __nv_bfloat162 pa = __floats2bfloat162_rn(p0, p1), pb = __floats2bfloat162_rn(p2, p3);
+                        packed[(i >> 1)] = *reinterpret_cast<uint32_t*>(&pa);
+                        packed[(i >> 1) + 1] = *reinterpret_cast<uint32_t*>(&pb);
+                    }
+                } else {
+#pragma unroll
+                    for (int i = 0; i < 16; ++i) packed[i] = 0u;
                 }
-                tmem_st16(s_addr + (c0 >> 1), packed);
+                tmem_st16p(s_addr + c * 16, packed);
+            }
+            {
+                float a0, a1, b0, b1;
+                unpack2(l2a, a0, a1);
+                unpack2(l2b, b0, b1);
+                l += (a0 + a1) + (b0 + b1);
             }
             tmem_wait_st();
             tc_fence_before();
