@@ -27,12 +27,9 @@ namespace pf {
 constexpr int BM = 128;             // query rows per CTA
 constexpr int BN = 128;             // key/value rows per tile
 constexpr int kBoxBytes = 128 * 128;  // one TMA box: 128 rows x 64 bf16 (128 bytes, swizzled)
-constexpr int kThreads = 160;
-constexpr uint32_t kSpinLimit = 1u << 22;
+constexpr uint32_t kSpinLimit = 1u << 26;
+constexpr uint64_t kWaitLimitNs = 1000000000ull;  // 1 s: far beyond any legitimate wait
 constexpr float kRescaleThreshold = 8.0f;  // log2 units
-
-// ---- barrier slots in shared memory
-enum { B_QFULL = 0, B_KFULL, B_VFULL, B_KEMPTY, B_VEMPTY, B_SFULL, B_PFULL, B_OFULL, B_COUNT };
 
 __device__ __forceinline__ uint32_t smem_u32(const void* p) { return (uint32_t)__cvta_generic_to_shared(p); }
 
@@ -60,12 +57,25 @@ __device__ __forceinline__ bool mbar_try_wait(uint32_t bar, uint32_t parity)
         : "memory");
     return ok != 0;
 }
-// Bounded wait.  Returns false when the limit ran out or another thread of the CTA gave up.
+__device__ __forceinline__ uint64_t global_ns()
+{
+    uint64_t t;
+    asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(t));
+    return t;
+}
+// Bounded wait: gives up after kWaitLimitNs of wall time (or kSpinLimit polls).  Returns false when
+// the limit ran out or another thread of the CTA gave up.
 __device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatile int* abort_flag, uint32_t* dev_status)
 {
+    uint64_t t0 = 0;
     for (uint32_t it = 0; it < kSpinLimit; ++it) {
         if (mbar_try_wait(bar, parity)) return true;
-        if ((it & 255u) == 255u && *abort_flag) return false;
+        if ((it & 63u) == 63u) {
+            if (*abort_flag) return false;
+            const uint64_t now = global_ns();
+            if (t0 == 0) t0 = now;
+            else if (now - t0 > kWaitLimitNs) break;
+        }
     }
     *abort_flag = 1;
     raise_status(dev_status, BT_DEV_TIMEOUT);
@@ -152,12 +162,6 @@ __device__ __forceinline__ void tmem_st32(uint32_t taddr, const float (&v)[32])
         : "memory");
 }
 
-struct Params {
-    void* out;
-    uint32_t* dev_status;
-    int T, n_qtiles;
-    float scale_log2;
-};
 
 // 16 consecutive 32-bit columns of this thread's TMEM lane (32 packed bf16).
 __device__ __forceinline__ void tmem_st16(uint32_t taddr, const uint32_t (&v)[16])
@@ -247,17 +251,106 @@ __device__ __forceinline__ float fmax3(float a, float b, float c)
     return d;
 }
 
+__device__ __forceinline__ uint64_t fadd2_rm(uint64_t a, uint64_t b)
+{
+    uint64_t d;
+    asm("add.rm.f32x2 %0, %1, %2;" : "=l"(d) : "l"(a), "l"(b));
+    return d;
+}
+// 2^x for two values on the FMA and integer pipes (no special-function unit): x = n + f with
+// n = floor(x), f in [0,1); 2^f by a cubic with maximum relative error 8.6e-5 (well below the bf16
+// rounding the result gets), then n is added to the exponent field.  x is clamped at -127 (result
+// 2^-127 flushes to 0 in the bf16 product); x must stay below 128.
+__device__ __forceinline__ void exp2_poly2(float x0, float x1, float& p0, float& p1)
+{
+    const float kMagic = 12582912.f;  // 1.5 * 2^23: adding it with round-down leaves floor(x) in the low mantissa bits
+    const uint64_t x = pack2(fmaxf(x0, -127.f), fmaxf(x1, -127.f));
+    const uint64_t t = fadd2_rm(x, pack2(kMagic, kMagic));
+    const uint64_t fl = fadd2(t, pack2(-kMagic, -kMagic));
+    const uint64_t f = ffma2(fl, pack2(-1.f, -1.f), x);
+    uint64_t q = ffma2(f, pack2(0.07706617563962936f, 0.07706617563962936f), pack2(0.22764593362808228f, 0.22764593362808228f));
+    q = ffma2(q, f, pack2(0.6951165795326233f, 0.6951165795326233f));
+    q = ffma2(q, f, pack2(1.f, 1.f));
+    float t0, t1, q0, q1;
+    unpack2(t, t0, t1);
+    unpack2(q, q0, q1);
+    p0 = __uint_as_float(__float_as_uint(q0) + (__float_as_uint(t0) << 23));
+    p1 = __uint_as_float(__float_as_uint(q1) + (__float_as_uint(t1) << 23));
+}
+
+// Work decomposition.  The T query blocks of one (sequence, head) form n = ceil(T/128) query tiles;
+// tile t needs key/value tiles 0..t.  An item is a pair of neighbouring query tiles taken from the
+// top: class k holds tiles A = n-1-2k (na = n-2k tile steps) and B = n-2-2k (nb = na-1 steps; absent
+// when A is tile 0).  The two tiles of an item walk the same key/value tiles, so K and V are loaded
+// once for both and their work is nearly equal, which keeps both softmax warpgroups busy.
+// Items are numbered item = bh * m + k (m = ceil(n/2) classes) and CTA c processes items c, c+G,
+// c+2G, ... with the grid size G coprime to m, so every CTA cycles through all classes (balanced
+// work) while the classes of one (sequence, head) run at the same time on neighbouring CTAs and
+// share its K and V through L2.
+struct Params {
+    void* out;
+    uint32_t* dev_status;
+    int T, n_qtiles, n_classes;
+    long long n_items;
+    float scale_log2;
+};
+
+// warps 0-3: softmax warpgroup of tile A, warps 4-7: of tile B
+constexpr int kProducerWarp = 8, kMmaWarp = 9;
+constexpr int kThreads = 320;
+constexpr int kKvStages = 2;
+#ifndef BT_PF_POLY_OF8
+#define BT_PF_POLY_OF8 0
+#endif
+#ifndef BT_PF_EARLY_CHUNKS
+#define BT_PF_EARLY_CHUNKS 3
+#endif
+constexpr int kPolyOf8 = BT_PF_POLY_OF8;                 // exponentials per 8 computed without the special-function unit (0,2,4,6,8)
+constexpr int kEarlyChunks = BT_PF_EARLY_CHUNKS;             // 32-column chunks of P signalled ahead of the rest
+constexpr int kQBufs = 3;                   // Q_A alternates between buffers 0 and 2, Q_B lives in buffer 1
+
+// barrier slots in shared memory
+enum {
+    B_QFULL = 0,                       // [kQBufs]  TMA -> MMA
+    B_QEMPTY = B_QFULL + kQBufs,       // [kQBufs]  MMA (commit) -> TMA
+    B_KFULL = B_QEMPTY + kQBufs,       // [kKvStages]
+    B_KEMPTY = B_KFULL + kKvStages,
+    B_VFULL = B_KEMPTY + kKvStages,
+    B_VEMPTY = B_VFULL + kKvStages,
+    B_SFULL = B_VEMPTY + kKvStages,    // [2] per query tile: S ready (and every earlier MMA done)
+    B_P0FULL = B_SFULL + 2,            // [2] per query tile: 128 softmax threads have written P columns 0..95
+    B_P1FULL = B_P0FULL + 2,           // [2] per query tile: ... and columns 96..127
+    B_OFULL = B_P1FULL + 2,            // [2] per query tile: last P V of the item done
+    B_COUNT = B_OFULL + 2
+};
+
 template <int HD>
 constexpr int smem_bytes()
 {
-    // Q, K, V tiles (HD/64 boxes each) + barriers, plus 1024 to align
-    return 1024 + (HD / 64) * kBoxBytes * 3 + 256;
+    // 3 Q tiles, 2 K and 2 V stages (HD/64 boxes each), barriers, plus 1024 to align
+    return 1024 + (HD / 64) * kBoxBytes * (kQBufs + 2 * kKvStages) + 256;
 }
 
-constexpr uint32_t kTmemCols = 256;  // S/P: 128 columns, O: up to 128 columns; two CTAs fit in the SM's 512
+constexpr uint32_t kTmemCols = 512;  // S_A, S_B (128 columns each), O_A, O_B (head_dim columns each)
+
+// The class-k item of a (sequence, head) with n query tiles.
+struct Item {
+    int bh, qa, qb, na, nb;  // qb = -1 and nb = 0 when the item has one tile only
+};
+__device__ __forceinline__ Item decode_item(long long item, const Params& p)
+{
+    Item it;
+    it.bh = (int)(item / p.n_classes);
+    const int k = (int)(item - (long long)it.bh * p.n_classes);
+    it.qa = p.n_qtiles - 1 - 2 * k;
+    it.qb = it.qa - 1;
+    it.na = it.qa + 1;
+    it.nb = it.qb + 1;  // 0 when qb == -1
+    return it;
+}
 
 template <int HD>
-__global__ void __launch_bounds__(kThreads, 2)
+__global__ void __launch_bounds__(kThreads, 1)
 block_prefill_tc_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_constant__ CUtensorMap mapK,
                         const __grid_constant__ CUtensorMap mapV, Params p)
 {
@@ -265,34 +358,25 @@ block_prefill_tc_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_c
     constexpr uint32_t TILE_BYTES = NB * kBoxBytes;
     constexpr uint32_t IDESC_S = make_idesc(BM, BN, false);
     constexpr uint32_t IDESC_O = make_idesc(BM, HD, true);
-    constexpr uint32_t COL_S = 0, COL_O = BN;   // TMEM columns: S (fp32) / P (bf16 pairs, in place) | O
+    // TMEM columns: S (fp32) / P (bf16 pairs, in place) of tiles A and B, then O of tiles A and B
+    constexpr uint32_t COL_S0 = 0, COL_O0 = 2 * BN;
 
     extern __shared__ uint8_t smem_raw[];
     const uint32_t base = (smem_u32(smem_raw) + 1023u) & ~1023u;
     uint8_t* gen_base = smem_raw + (base - smem_u32(smem_raw));
-    const uint32_t sQ = base;
-    const uint32_t sK = sQ + TILE_BYTES;
-    const uint32_t sV = sK + TILE_BYTES;
-    const uint32_t sBar = sV + TILE_BYTES;      // B_COUNT x 8 bytes
+    const uint32_t sQ = base;                               // kQBufs tiles
+    const uint32_t sK = sQ + kQBufs * TILE_BYTES;           // kKvStages tiles
+    const uint32_t sV = sK + kKvStages * TILE_BYTES;        // kKvStages tiles
+    const uint32_t sBar = sV + kKvStages * TILE_BYTES;      // B_COUNT x 8 bytes
     uint8_t* gen_tail = gen_base + (sBar - base);
     uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(gen_tail + B_COUNT * 8);
     volatile int* abort_flag = reinterpret_cast<volatile int*>(gen_tail + B_COUNT * 8 + 8);
     auto bar = [&](int i) { return sBar + 8u * i; };
 
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-    const int bh = blockIdx.x / p.n_qtiles;
-    const int qt = p.n_qtiles - 1 - (blockIdx.x - bh * p.n_qtiles);  // heaviest query tiles first
-    const int n_kv = qt + 1;                                          // tiles 0 .. diagonal
 
     if (threadIdx.x == 0) {
-        mbar_init(bar(B_QFULL), 1);
-        mbar_init(bar(B_KFULL), 1);
-        mbar_init(bar(B_VFULL), 1);
-        mbar_init(bar(B_KEMPTY), 1);
-        mbar_init(bar(B_VEMPTY), 1);
-        mbar_init(bar(B_SFULL), 1);
-        mbar_init(bar(B_PFULL), 128);
-        mbar_init(bar(B_OFULL), 1);
+        for (int i = 0; i < B_COUNT; ++i) mbar_init(bar(i), (i >= B_P0FULL && i < B_P0FULL + 4) ? 128u : 1u);
         *abort_flag = 0;
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     }
@@ -305,193 +389,273 @@ block_prefill_tc_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_c
     tc_fence_after();
     const uint32_t tmem = *tmem_slot;
 
-    if (warp == 4) {
-        // ------------------------------------------------------------------ TMA producer + MMA issuer
+    if (warp == kProducerWarp) {
+        // ------------------------------------------------------------------ TMA producer
         if (lane == 0) {
             asm volatile("prefetch.tensormap [%0];" ::"l"(&mapQ) : "memory");
             asm volatile("prefetch.tensormap [%0];" ::"l"(&mapK) : "memory");
             asm volatile("prefetch.tensormap [%0];" ::"l"(&mapV) : "memory");
-            auto load_k = [&](int j) {
-                mbar_expect_tx(bar(B_KFULL), TILE_BYTES);
-                for (int bx = 0; bx < NB; ++bx) tma_load_3d(sK + bx * kBoxBytes, &mapK, bar(B_KFULL), bx * 64, j * BN, bh);
-            };
-            auto load_v = [&](int j) {
-                mbar_expect_tx(bar(B_VFULL), TILE_BYTES);
-                for (int bx = 0; bx < NB; ++bx) tma_load_3d(sV + bx * kBoxBytes, &mapV, bar(B_VFULL), bx * 64, j * BN, bh);
-            };
-            // S_j = Q K_j^T.  It overwrites the columns P_{j-1} lived in: MMAs of one thread execute in
-            // issue order, and P_{j-1} V_{j-1} is always issued before S_j.
-            auto issue_s = [&]() {
-#pragma unroll
-                for (int kk = 0; kk < HD / 16; ++kk) {
-                    const uint32_t off = (kk >> 2) * kBoxBytes + (kk & 3) * 32;
-                    mma_bf16(tmem + COL_S, make_desc(sQ + off, 16, 1024), make_desc(sK + off, 16, 1024), IDESC_S, kk > 0 ? 1u : 0u);
-                }
-                mma_commit(bar(B_SFULL));
-                mma_commit(bar(B_KEMPTY));
-            };
-            mbar_expect_tx(bar(B_QFULL), TILE_BYTES);
-            for (int bx = 0; bx < NB; ++bx) tma_load_3d(sQ + bx * kBoxBytes, &mapQ, bar(B_QFULL), bx * 64, qt * BM, bh);
-            load_k(0);
-            load_v(0);
-            bool ok = mbar_wait(bar(B_QFULL), 0, abort_flag, p.dev_status) &&
-                      mbar_wait(bar(B_KFULL), 0, abort_flag, p.dev_status);
-            if (ok) {
-                tc_fence_after();
-                issue_s();
-            }
-            for (int j = 0; ok && j < n_kv; ++j) {
-                const bool more = j + 1 < n_kv;
-                if (more) {  // K_{j+1} may land once S_j has consumed K_j
-                    ok = mbar_wait(bar(B_KEMPTY), j & 1, abort_flag, p.dev_status);
+            // n-th use of a buffer: wait for its EMPTY barrier with parity (n & 1) ^ 1 (passes at once
+            // on a fresh barrier), then fill it; the consumer waits FULL with parity n & 1.
+            uint32_t q_uses[kQBufs] = {0, 0, 0};
+            uint32_t kv_count = 0;   // key/value tiles loaded so far (K and V advance together)
+            uint32_t n_done = 0;     // items processed by this CTA
+            bool ok = true;
+            for (long long item = blockIdx.x; ok && item < p.n_items; item += gridDim.x, ++n_done) {
+                const Item it = decode_item(item, p);
+                auto load_q = [&](int buf, int qt) {
+                    ok = ok && mbar_wait(bar(B_QEMPTY + buf), (q_uses[buf] & 1) ^ 1, abort_flag, p.dev_status);
+                    if (!ok) return;
+                    ++q_uses[buf];
+                    mbar_expect_tx(bar(B_QFULL + buf), TILE_BYTES);
+                    for (int bx = 0; bx < NB; ++bx)
+                        tma_load_3d(sQ + buf * TILE_BYTES + bx * kBoxBytes, &mapQ, bar(B_QFULL + buf), bx * 64, qt * BM, it.bh);
+                };
+                load_q((n_done & 1) ? 2 : 0, it.qa);
+                if (it.nb > 0) load_q(1, it.qb);
+                for (int j = 0; ok && j < it.na; ++j, ++kv_count) {
+                    const uint32_t st = kv_count % kKvStages, par = ((kv_count / kKvStages) & 1) ^ 1;
+                    ok = mbar_wait(bar(B_KEMPTY + st), par, abort_flag, p.dev_status);
                     if (!ok) break;
-                    load_k(j + 1);
+                    mbar_expect_tx(bar(B_KFULL + st), TILE_BYTES);
+                    for (int bx = 0; bx < NB; ++bx)
+                        tma_load_3d(sK + st * TILE_BYTES + bx * kBoxBytes, &mapK, bar(B_KFULL + st), bx * 64, j * BN, it.bh);
+                    ok = mbar_wait(bar(B_VEMPTY + st), par, abort_flag, p.dev_status);
+                    if (!ok) break;
+                    mbar_expect_tx(bar(B_VFULL + st), TILE_BYTES);
+                    for (int bx = 0; bx < NB; ++bx)
+                        tma_load_3d(sV + st * TILE_BYTES + bx * kBoxBytes, &mapV, bar(B_VFULL + st), bx * 64, j * BN, it.bh);
                 }
-                ok = mbar_wait(bar(B_PFULL), j & 1, abort_flag, p.dev_status) &&
-                     mbar_wait(bar(B_VFULL), j & 1, abort_flag, p.dev_status);
-                if (!ok) break;
-                tc_fence_after();
+            }
+        }
+    } else if (warp == kMmaWarp) {
+        // ------------------------------------------------------------------ MMA issuer
+        // Issue order per item (tile A has one more step than tile B):
+        //   S_A(0) S_B(0) | PV_A(0) S_A(1) PV_B(0) S_B(1) | PV_A(1) S_A(2) PV_B(1) S_B(2) | ...
+        // so the tensor pipe works on one tile while the other tile's warpgroup does its softmax.
+        // S_x(j+1) overwrites the columns P_x(j) lived in: MMAs of one thread execute in issue order
+        // and P_x(j) V(j) is always issued before S_x(j+1).
+        if (lane == 0) {
+            uint32_t q_uses[kQBufs] = {0, 0, 0};
+            uint32_t kv_base = 0;                 // key/value tiles consumed by earlier items
+            uint32_t p_count[2] = {0, 0};         // P tiles consumed so far, per query tile slot
+            uint32_t n_done = 0;
+            bool ok = true;
+            for (long long item = blockIdx.x; ok && item < p.n_items; item += gridDim.x, ++n_done) {
+                const Item it = decode_item(item, p);
+                const int qbuf[2] = {(n_done & 1) ? 2 : 0, 1};
+                const int steps[2] = {it.na, it.nb};
+                // S_x(j) = Q_x K_j^T, then the barriers that fire when it (and all before it) is done
+                auto issue_s = [&](int x, int j) {
+                    const uint32_t kc = kv_base + j, st = kc % kKvStages;
+                    ok = ok && mbar_wait(bar(B_KFULL + st), (kc / kKvStages) & 1, abort_flag, p.dev_status);
+                    if (ok && j == 0) {
+                        ok = mbar_wait(bar(B_QFULL + qbuf[x]), q_uses[qbuf[x]] & 1, abort_flag, p.dev_status);
+                        ++q_uses[qbuf[x]];
+                    }
+                    if (!ok) return;
+                    tc_fence_after();
+                    const uint32_t q0 = sQ + qbuf[x] * TILE_BYTES, k0 = sK + st * TILE_BYTES;
 #pragma unroll
-                for (int kk = 0; kk < BN / 16; ++kk) {
+                    for (int kk = 0; kk < HD / 16; ++kk) {
+                        const uint32_t off = (kk >> 2) * kBoxBytes + (kk & 3) * 32;
+                        mma_bf16(tmem + COL_S0 + x * BN, make_desc(q0 + off, 16, 1024), make_desc(k0 + off, 16, 1024), IDESC_S,
+                                 kk > 0 ? 1u : 0u);
+                    }
+                    mma_commit(bar(B_SFULL + x));
+                    if (j == steps[x] - 1) mma_commit(bar(B_QEMPTY + qbuf[x]));  // last use of this Q tile
+                    // K_j is free after its last reader: tile B while it still runs, else tile A
+                    if (x == 1 || j >= it.nb) mma_commit(bar(B_KEMPTY + st));
+                };
+                // O_x (+)= P_x(j) V_j
+                auto issue_pv = [&](int x, int j) {
+                    const uint32_t kc = kv_base + j, st = kc % kKvStages;
+                    ok = ok && mbar_wait(bar(B_P0FULL + x), p_count[x] & 1, abort_flag, p.dev_status) &&
+                         mbar_wait(bar(B_VFULL + st), (kc / kKvStages) & 1, abort_flag, p.dev_status);
+                    if (!ok) return;
+                    tc_fence_after();
+                    const uint32_t v0 = sV + st * TILE_BYTES;
                     // A = P from tensor memory: 16 kv columns = 8 packed 32-bit columns;
                     // B = V, MN-major: 16 kv rows = 2048 bytes; next 64 head dims one box further
-                    mma_bf16_ts(tmem + COL_O, tmem + COL_S + kk * 8, make_desc(sV + kk * 2048, kBoxBytes, 1024), IDESC_O,
-                                (j > 0 || kk > 0) ? 1u : 0u);
+                    auto pv = [&](int kk) {
+                        mma_bf16_ts(tmem + COL_O0 + x * HD, tmem + COL_S0 + x * BN + kk * 8, make_desc(v0 + kk * 2048, kBoxBytes, 1024),
+                                    IDESC_O, (j > 0 || kk > 0) ? 1u : 0u);
+                    };
+                    // the first three quarters of P arrive early: their share of the product runs while
+                    // the softmax warps still work on the last quarter
+#pragma unroll
+                    for (int kk = 0; kk < kEarlyChunks * 2; ++kk) pv(kk);
+                    ok = mbar_wait(bar(B_P1FULL + x), p_count[x] & 1, abort_flag, p.dev_status);
+                    if (!ok) return;
+                    ++p_count[x];
+                    tc_fence_after();
+#pragma unroll
+                    for (int kk = kEarlyChunks * 2; kk < BN / 16; ++kk) pv(kk);
+                    if (x == 1 || j >= it.nb) mma_commit(bar(B_VEMPTY + st));
+                    if (j == steps[x] - 1) mma_commit(bar(B_OFULL + x));
+                };
+                issue_s(0, 0);
+                if (it.nb > 0) issue_s(1, 0);
+                for (int j = 0; ok && j < it.na; ++j) {
+                    issue_pv(0, j);
+                    if (j + 1 < it.na) issue_s(0, j + 1);
+                    if (j < it.nb) {
+                        issue_pv(1, j);
+                        if (j + 1 < it.nb) issue_s(1, j + 1);
+                    }
                 }
-                mma_commit(bar(B_VEMPTY));
-                if (!more) {
-                    mma_commit(bar(B_OFULL));
-                    break;
-                }
-                // queue S_{j+1} behind P_j V_j so the tensor pipe never waits for this thread
-                ok = mbar_wait(bar(B_KFULL), (j + 1) & 1, abort_flag, p.dev_status);
-                if (!ok) break;
-                tc_fence_after();
-                issue_s();
-                // V_{j+1} may land once P_j V_j has consumed V_j
-                ok = mbar_wait(bar(B_VEMPTY), j & 1, abort_flag, p.dev_status);
-                if (!ok) break;
-                load_v(j + 1);
+                kv_base += it.na;
             }
         }
     } else {
         // ------------------------------------------------------------------ softmax: thread = query row
-        const int row = threadIdx.x;                       // TMEM lane
-        const int grow = qt * BM + row;                    // query block index within the sequence
-        const uint32_t lane_base = tmem + ((uint32_t)(warp * 32) << 16);
-        float m_ref = kNegInf, l = 0.f;
+        const int x = warp >> 2;                           // 0: tile A (warps 0-3), 1: tile B (warps 4-7)
+        const int wq = warp & 3;                           // TMEM lane quarter this warp may access
+        const int row = wq * 32 + lane;                    // TMEM lane = query row within the tile
+        const uint32_t lane_base = tmem + ((uint32_t)(wq * 32) << 16);
+        const uint32_t s_addr = lane_base + COL_S0 + x * BN;
+        const uint32_t o_addr = lane_base + COL_O0 + x * HD;
+        uint32_t s_count = 0, o_count = 0;                 // S tiles / O tiles consumed so far by this thread
         bool ok = true;
-        for (int j = 0; j < n_kv; ++j) {
-            const bool diag = (j == qt);
-            ok = mbar_wait(bar(B_SFULL), j & 1, abort_flag, p.dev_status);  // S_j ready; O settled (all earlier MMAs done)
-            if (!ok) break;
-            tc_fence_after();
-            const uint32_t s_addr = lane_base + COL_S;
-            // On the diagonal tile the rows of warp w (32w .. 32w+31) see nothing right of column
-            // 32w+31: only column chunks 0..w are loaded and exponentiated, chunk w with a per-row mask.
-            const int nch = diag ? warp + 1 : BN / 32;
-            uint32_t sr[BN];
-#pragma unroll
-            for (int c = 0; c < BN / 32; ++c)
-                if (c < nch) tmem_ld32_issue(s_addr + c * 32, sr + c * 32);
-            tmem_wait_ld();
-#pragma unroll
-            for (int c = 0; c < BN / 32; ++c)
-                if (c < nch) tmem_ld_fence32(sr + c * 32);
-            if (diag) {  // masked scores become -inf: they drop out of the maximum and exponentiate to 0
+        for (long long item = blockIdx.x; ok && item < p.n_items; item += gridDim.x) {
+            const Item it = decode_item(item, p);
+            const int qt = x ? it.qb : it.qa, n_kv = x ? it.nb : it.na;
+            if (n_kv == 0) continue;                       // single-tile item: warpgroup B has nothing to do
+            const int grow = qt * BM + row;                // query block index within the sequence
+            float m_ref = kNegInf, l = 0.f;
+            for (int j = 0; j < n_kv; ++j, ++s_count) {
+                const bool diag = (j == qt);
+                ok = mbar_wait(bar(B_SFULL + x), s_count & 1, abort_flag, p.dev_status);  // S_j ready; O settled
+                if (!ok) break;
+                tc_fence_after();
+                // On the diagonal tile the rows of warp w (32w .. 32w+31) see nothing right of column
+                // 32w+31: only column chunks 0..w are loaded and exponentiated, chunk w with a per-row mask.
+                const int nch = diag ? wq + 1 : BN / 32;
+                uint32_t sr[BN];
 #pragma unroll
                 for (int c = 0; c < BN / 32; ++c)
-                    if (c == warp) {
+                    if (c < nch) tmem_ld32_issue(s_addr + c * 32, sr + c * 32);
+                tmem_wait_ld();
 #pragma unroll
-                        for (int i = 0; i < 32; ++i)
-                            if (i > lane) sr[c * 32 + i] = __float_as_uint(kNegInf);
-                    }
-            }
-            float mx = kNegInf;
+                for (int c = 0; c < BN / 32; ++c)
+                    if (c < nch) tmem_ld_fence32(sr + c * 32);
+                if (diag) {  // masked scores become -inf: they drop out of the maximum and exponentiate to 0
 #pragma unroll
-            for (int c = 0; c < BN / 32; ++c)
-                if (c < nch) {
+                    for (int c = 0; c < BN / 32; ++c)
+                        if (c == wq) {
 #pragma unroll
-                    for (int i = 0; i < 32; i += 2)
-                        mx = fmax3(mx, __uint_as_float(sr[c * 32 + i]), __uint_as_float(sr[c * 32 + i + 1]));
+                            for (int i = 0; i < 32; ++i)
+                                if (i > lane) sr[c * 32 + i] = __float_as_uint(kNegInf);
+                        }
                 }
-            mx *= p.scale_log2;
-            float factor = 1.f;
-            const bool grow_ref = mx > m_ref + kRescaleThreshold;  // first tile: m_ref = -inf
-            if (grow_ref) {
-                factor = (m_ref == kNegInf) ? 0.f : ex2(m_ref - mx);
-                m_ref = mx;
-            }
-            if (j > 0) {
-                if (__any_sync(0xffffffffu, grow_ref)) {
+                float mx4[4] = {kNegInf, kNegInf, kNegInf, kNegInf};  // independent chains: the maximum is latency-bound
+#pragma unroll
+                for (int c = 0; c < BN / 32; ++c)
+                    if (c < nch) {
+#pragma unroll
+                        for (int i = 0; i < 32; i += 8) {
+#pragma unroll
+                            for (int u = 0; u < 4; ++u)
+                                mx4[u] = fmax3(mx4[u], __uint_as_float(sr[c * 32 + i + 2 * u]), __uint_as_float(sr[c * 32 + i + 2 * u + 1]));
+                        }
+                    }
+                float mx = fmaxf(fmaxf(mx4[0], mx4[1]), fmaxf(mx4[2], mx4[3]));
+                mx *= p.scale_log2;
+                float factor = 1.f;
+                const bool grow_ref = mx > m_ref + kRescaleThreshold;  // first tile: m_ref = -inf
+                if (grow_ref) {
+                    factor = (m_ref == kNegInf) ? 0.f : ex2(m_ref - mx);
+                    m_ref = mx;
+                }
+                if (j > 0) {
+                    if (__any_sync(0xffffffffu, grow_ref)) {
 #pragma unroll 1
-                    for (int c0 = 0; c0 < HD; c0 += 32) {
-                        float o[32];
-                        tmem_ld32(lane_base + COL_O + c0, o);
+                        for (int c0 = 0; c0 < HD; c0 += 32) {
+                            float o[32];
+                            tmem_ld32(o_addr + c0, o);
 #pragma unroll
-                        for (int i = 0; i < 32; ++i) o[i] *= factor;
-                        tmem_st32(lane_base + COL_O + c0, o);
+                            for (int i = 0; i < 32; ++i) o[i] *= factor;
+                            tmem_st32(o_addr + c0, o);
+                        }
+                    }
+                    l *= factor;
+                }
+                // P = 2^(s*scale - m_ref) as bf16 pairs over the S columns (chunk c of P lands in columns
+                // 16c .. 16c+15; every S column is already in registers).  The row sum is taken in fp32
+                // before the rounding: the rounding errors of the 128 terms average out in the normaliser.
+                const uint64_t sc2 = pack2(p.scale_log2, p.scale_log2), nm2 = pack2(-m_ref, -m_ref);
+                uint64_t l2a = pack2(0.f, 0.f), l2b = l2a;
+#pragma unroll
+                for (int c = 0; c < BN / 32; ++c) {
+                    uint32_t packed[16];
+                    if (c < nch) {
+#pragma unroll
+                        for (int i = 0; i < 32; i += 4) {
+                            const uint32_t* e = sr + c * 32 + i;
+                            float x0, x1, x2, x3;
+                            unpack2(ffma2(pack2(__uint_as_float(e[0]), __uint_as_float(e[1])), sc2, nm2), x0, x1);
+                            unpack2(ffma2(pack2(__uint_as_float(e[2]), __uint_as_float(e[3])), sc2, nm2), x2, x3);
+                            // kPolyOf8 of every 8 exponentials go to the FMA pipes, the rest to the
+                            // special-function unit (16 per clock per SM, as busy as the tensor pipe here)
+                            float p0, p1, p2, p3;
+                            if ((i & 4) ? (kPolyOf8 >= 4) : (kPolyOf8 >= 2)) exp2_poly2(x0, x1, p0, p1);
+                            else { p0 = ex2(x0); p1 = ex2(x1); }
+                            if ((i & 4) ? (kPolyOf8 >= 8) : (kPolyOf8 >= 6)) exp2_poly2(x2, x3, p2, p3);
+                            else { p2 = ex2(x2); p3 = ex2(x3); }
+                            l2a = fadd2(l2a, pack2(p0, p1));
+                            l2b = fadd2(l2b, pack2(p2, p3));
+                            __nv_bfloat162 pa = __floats2bfloat162_rn(p0, p1), pb = __floats2bfloat162_rn(p2, p3);
+                            packed[(i >> 1)] = *reinterpret_cast<uint32_t*>(&pa);
+                            packed[(i >> 1) + 1] = *reinterpret_cast<uint32_t*>(&pb);
+                        }
+                    } else {
+#pragma unroll
+                        for (int i = 0; i < 16; ++i) packed[i] = 0u;
+                    }
+                    tmem_st16p(s_addr + c * 16, packed);
+                    if (c == kEarlyChunks - 1) {  // columns 0..95 of P are in place: let their share of P V start
+                        tmem_wait_st();
+                        tc_fence_before();
+                        mbar_arrive(bar(B_P0FULL + x));
                     }
                 }
-                l *= factor;
-            }
-            // P = 2^(s*scale - m_ref) as bf16 pairs over the S columns (chunk c of P lands in columns
-            // 16c .. 16c+15; every S column is already in registers).  The row sum is taken in fp32
-            // before the rounding: the rounding errors of the 128 terms average out in the normaliser.
-            const uint64_t sc2 = pack2(p.scale_log2, p.scale_log2), nm2 = pack2(-m_ref, -m_ref);
-            uint64_t l2a = pack2(0.f, 0.f), l2b = l2a;
-#pragma unroll
-            for (int c = 0; c < BN / 32; ++c) {
-                uint32_t packed[16];
-                if (c < nch) {
-#pragma unroll
-                    for (int i = 0; i < 32; i += 4) {
-                        const uint32_t* e = sr + c * 32 + i;
-                        float x0, x1, x2, x3;
-                        unpack2(ffma2(pack2(__uint_as_float(e[0]), __uint_as_float(e[1])), sc2, nm2), x0, x1);
-                        unpack2(ffma2(pack2(__uint_as_float(e[2]), __uint_as_float(e[3])), sc2, nm2), x2, x3);
-                        const float p0 = ex2(x0), p1 = ex2(x1), p2 = ex2(x2), p3 = ex2(x3);
-                        l2a = fadd2(l2a, pack2(p0, p1));
-                        l2b = fadd2(l2b, pack2(p2, p3));
-                        __nv_bfloat162 pa = __floats2bfloat162_rn(p0, p1), pb = __floats2bfloat162_rn(p2, p3);
-                        packed[(i >> 1)] = *reinterpret_cast<uint32_t*>(&pa);
-                        packed[(i >> 1) + 1] = *reinterpret_cast<uint32_t*>(&pb);
-                    }
-                } else {
-#pragma unroll
-                    for (int i = 0; i < 16; ++i) packed[i] = 0u;
+                {
+                    float a0, a1, b0, b1;
+                    unpack2(l2a, a0, a1);
+                    unpack2(l2b, b0, b1);
+                    l += (a0 + a1) + (b0 + b1);
                 }
-                tmem_st16p(s_addr + c * 16, packed);
+                tmem_wait_st();
+                tc_fence_before();
+                mbar_arrive(bar(B_P1FULL + x));
             }
-            {
-                float a0, a1, b0, b1;
-                unpack2(l2a, a0, a1);
-                unpack2(l2b, b0, b1);
-                l += (a0 + a1) + (b0 + b1);
-            }
-            tmem_wait_st();
-            tc_fence_before();
-            mbar_arrive(bar(B_PFULL));
-        }
-        if (ok) ok = mbar_wait(bar(B_OFULL), 0, abort_flag, p.dev_status);
-        if (ok) {
+            if (ok) ok = mbar_wait(bar(B_OFULL + x), o_count & 1, abort_flag, p.dev_status);
+            ++o_count;
+            if (!ok) break;
             tc_fence_after();
             const float inv = l > 0.f ? 1.f / l : 0.f;
-            bf16* orow = reinterpret_cast<bf16*>(p.out) + ((size_t)bh * p.T + grow) * HD;
+            bf16* orow = reinterpret_cast<bf16*>(p.out) + ((size_t)it.bh * p.T + grow) * HD;
 #pragma unroll 1
-            for (int c0 = 0; c0 < HD; c0 += 32) {
-                float o[32];
-                tmem_ld32(lane_base + COL_O + c0, o);
+            for (int c0 = 0; c0 < HD; c0 += 64) {
+                uint32_t o[64];
+                tmem_ld32_issue(o_addr + c0, o);
+                tmem_ld32_issue(o_addr + c0 + 32, o + 32);
+                tmem_wait_ld();
+                tmem_ld_fence32(o);
+                tmem_ld_fence32(o + 32);
                 if (grow < p.T) {
 #pragma unroll
-                    for (int q8 = 0; q8 < 4; ++q8) {
+                    for (int q8 = 0; q8 < 8; ++q8) {
                         float f[8];
 #pragma unroll
-                        for (int i = 0; i < 8; ++i) f[i] = o[q8 * 8 + i] * inv;
+                        for (int i = 0; i < 8; ++i) f[i] = __uint_as_float(o[q8 * 8 + i]) * inv;
                         *reinterpret_cast<uint4*>(orow + c0 + q8 * 8) = pack8(f);
                     }
                 }
             }
+            // the next item's first P V overwrites O: it is issued only after this thread's next
+            // arrival on PFULL, which follows these loads in program order
+            tc_fence_before();
         }
     }
 
@@ -538,15 +702,32 @@ static bool make_map(CUtensorMap* m, const void* ptr, int hd, int rows, long lon
               CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
 }
 
+static int gcd_int(int a, int b)
+{
+    while (b) {
+        int t = a % b;
+        a = b;
+        b = t;
+    }
+    return a;
+}
+
 template <int HD>
 static cudaError_t launch_t(const PrefillArgs& a, uint32_t* dev_status, cudaStream_t stream)
 {
-    static bool attr_set = false;
-    if (!attr_set) {
-        cudaError_t e = cudaFuncSetAttribute(block_prefill_tc_kernel<HD>, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                                             smem_bytes<HD>());
+    constexpr int kMaxDevices = 64;
+    static int sm_count[kMaxDevices];  // 0 = this device has not been set up yet
+    int dev = 0;
+    cudaError_t e = cudaGetDevice(&dev);
+    if (e != cudaSuccess) return e;
+    if (dev < 0 || dev >= kMaxDevices) return cudaErrorInvalidDevice;
+    if (!sm_count[dev]) {
+        e = cudaFuncSetAttribute(block_prefill_tc_kernel<HD>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem_bytes<HD>());
         if (e != cudaSuccess) return e;
-        attr_set = true;
+        int n = 0;
+        e = cudaDeviceGetAttribute(&n, cudaDevAttrMultiProcessorCount, dev);
+        if (e != cudaSuccess) return e;
+        sm_count[dev] = n > 0 ? n : 1;
     }
     const long long slabs = (long long)a.B * a.H;
     CUtensorMap mq, mk, mv;
@@ -558,10 +739,14 @@ static cudaError_t launch_t(const PrefillArgs& a, uint32_t* dev_status, cudaStre
     p.dev_status = dev_status;
     p.T = a.T;
     p.n_qtiles = (a.T + BM - 1) / BM;
+    p.n_classes = (p.n_qtiles + 1) / 2;
+    p.n_items = slabs * p.n_classes;
     p.scale_log2 = a.scale_log2;
-    const long long ctas = slabs * p.n_qtiles;
-    if (ctas > 0x7fffffffLL) return cudaErrorInvalidConfiguration;
-    block_prefill_tc_kernel<HD><<<(unsigned)ctas, kThreads, smem_bytes<HD>(), stream>>>(mq, mk, mv, p);
+    // one persistent CTA per SM; a grid size coprime to the number of classes makes every CTA
+    // cycle through all classes (heavy and light items alike)
+    long long grid = p.n_items < sm_count[dev] ? p.n_items : sm_count[dev];
+    while (grid > 1 && p.n_items > grid && gcd_int((int)grid, p.n_classes) != 1) --grid;
+    block_prefill_tc_kernel<HD><<<(unsigned)grid, kThreads, smem_bytes<HD>(), stream>>>(mq, mk, mv, p);
     return cudaGetLastError();
 }
 
