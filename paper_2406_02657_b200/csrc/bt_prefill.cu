@@ -90,6 +90,14 @@ __device__ __forceinline__ void tma_load_3d(uint32_t dst, const CUtensorMap* map
         : "memory");
 }
 
+// Tile store shared -> global (rows outside the tensor are dropped), as one bulk group of this thread.
+__device__ __forceinline__ void tma_store_3d(const CUtensorMap* map, uint32_t src, int c0, int c1, int c2)
+{
+    asm volatile("cp.async.bulk.tensor.3d.global.shared::cta.bulk_group [%0, {%2, %3, %4}], [%1];"
+                 ::"l"(map), "r"(src), "r"(c0), "r"(c1), "r"(c2)
+                 : "memory");
+}
+
 // Shared-memory matrix descriptor, 128-byte swizzle (layout type 2), descriptor version 1.
 __device__ __forceinline__ uint64_t make_desc(uint32_t saddr, uint32_t lbo_bytes, uint32_t sbo_bytes)
 {
@@ -288,7 +296,6 @@ __device__ __forceinline__ void exp2_poly2(float x0, float x1, float& p0, float&
 // work) while the classes of one (sequence, head) run at the same time on neighbouring CTAs and
 // share its K and V through L2.
 struct Params {
-    void* out;
     uint32_t* dev_status;
     int T, n_qtiles, n_classes;
     long long n_items;
@@ -352,7 +359,7 @@ __device__ __forceinline__ Item decode_item(long long item, const Params& p)
 template <int HD>
 __global__ void __launch_bounds__(kThreads, 1)
 block_prefill_tc_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_constant__ CUtensorMap mapK,
-                        const __grid_constant__ CUtensorMap mapV, Params p)
+                        const __grid_constant__ CUtensorMap mapV, const __grid_constant__ CUtensorMap mapO, Params p)
 {
     constexpr int NB = HD / 64;                 // TMA boxes per operand tile
     constexpr uint32_t TILE_BYTES = NB * kBoxBytes;
@@ -395,6 +402,7 @@ block_prefill_tc_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_c
             asm volatile("prefetch.tensormap [%0];" ::"l"(&mapQ) : "memory");
             asm volatile("prefetch.tensormap [%0];" ::"l"(&mapK) : "memory");
             asm volatile("prefetch.tensormap [%0];" ::"l"(&mapV) : "memory");
+            asm volatile("prefetch.tensormap [%0];" ::"l"(&mapO) : "memory");
             // n-th use of a buffer: wait for its EMPTY barrier with parity (n & 1) ^ 1 (passes at once
             // on a fresh barrier), then fill it; the consumer waits FULL with parity n & 1.
             uint32_t q_uses[kQBufs] = {0, 0, 0};
@@ -491,7 +499,10 @@ block_prefill_tc_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_c
                     tc_fence_after();
 #pragma unroll
                     for (int kk = kEarlyChunks * 2; kk < BN / 16; ++kk) pv(kk);
-                    if (x == 1 || j >= it.nb) mma_commit(bar(B_VEMPTY + st));
+                    // V_j is free after its last reader (tile B while it still runs, else tile A) - except the
+                    // last V tile of each query tile: its stage stages that tile's output first and is
+                    // released by the epilogue
+                    if ((x == 1 || j >= it.nb) && j != steps[x] - 1) mma_commit(bar(B_VEMPTY + st));
                     if (j == steps[x] - 1) mma_commit(bar(B_OFULL + x));
                 };
                 issue_s(0, 0);
@@ -516,12 +527,14 @@ block_prefill_tc_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_c
         const uint32_t s_addr = lane_base + COL_S0 + x * BN;
         const uint32_t o_addr = lane_base + COL_O0 + x * HD;
         uint32_t s_count = 0, o_count = 0;                 // S tiles / O tiles consumed so far by this thread
+        uint32_t kv_base = 0;                              // key/value tiles consumed by earlier items
         bool ok = true;
         for (long long item = blockIdx.x; ok && item < p.n_items; item += gridDim.x) {
             const Item it = decode_item(item, p);
             const int qt = x ? it.qb : it.qa, n_kv = x ? it.nb : it.na;
+            const uint32_t stage_o = (kv_base + n_kv - 1) % kKvStages;  // stage of this tile's last V tile
+            kv_base += it.na;
             if (n_kv == 0) continue;                       // single-tile item: warpgroup B has nothing to do
-            const int grow = qt * BM + row;                // query block index within the sequence
             float m_ref = kNegInf, l = 0.f;
             for (int j = 0; j < n_kv; ++j, ++s_count) {
                 const bool diag = (j == qt);
@@ -589,19 +602,27 @@ block_prefill_tc_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_c
                 for (int c = 0; c < BN / 32; ++c) {
                     uint32_t packed[16];
                     if (c < nch) {
+                        // three passes over the chunk, in place, so that 32 independent exponentials are in flight
+#pragma unroll
+                        for (int i = 0; i < 32; i += 2) {
+                            float x0, x1;
+                            unpack2(ffma2(pack2(__uint_as_float(sr[c * 32 + i]), __uint_as_float(sr[c * 32 + i + 1])), sc2, nm2), x0, x1);
+                            sr[c * 32 + i] = __float_as_uint(x0);
+                            sr[c * 32 + i + 1] = __float_as_uint(x1);
+                        }
+#pragma unroll
+                        for (int i = 0; i < 32; i += 2) {
+                            // kPolyOf8 of every 8 exponentials go to the FMA pipes, the rest to the special-function unit
+                            float p0, p1;
+                            if (((i >> 1) & 3) < kPolyOf8 / 2) exp2_poly2(__uint_as_float(sr[c * 32 + i]), __uint_as_float(sr[c * 32 + i + 1]), p0, p1);
+                            else { p0 = ex2(__uint_as_float(sr[c * 32 + i])); p1 = ex2(__uint_as_float(sr[c * 32 + i + 1])); }
+                            sr[c * 32 + i] = __float_as_uint(p0);
+                            sr[c * 32 + i + 1] = __float_as_uint(p1);
+                        }
 #pragma unroll
                         for (int i = 0; i < 32; i += 4) {
-                            const uint32_t* e = sr + c * 32 + i;
-                            float x0, x1, x2, x3;
-                            unpack2(ffma2(pack2(__uint_as_float(e[0]), __uint_as_float(e[1])), sc2, nm2), x0, x1);
-                            unpack2(ffma2(pack2(__uint_as_float(e[2]), __uint_as_float(e[3])), sc2, nm2), x2, x3);
-                            // kPolyOf8 of every 8 exponentials go to the FMA pipes, the rest to the
-                            // special-function unit (16 per clock per SM, as busy as the tensor pipe here)
-                            float p0, p1, p2, p3;
-                            if ((i & 4) ? (kPolyOf8 >= 4) : (kPolyOf8 >= 2)) exp2_poly2(x0, x1, p0, p1);
-                            else { p0 = ex2(x0); p1 = ex2(x1); }
-                            if ((i & 4) ? (kPolyOf8 >= 8) : (kPolyOf8 >= 6)) exp2_poly2(x2, x3, p2, p3);
-                            else { p2 = ex2(x2); p3 = ex2(x3); }
+                            const float p0 = __uint_as_float(sr[c * 32 + i]), p1 = __uint_as_float(sr[c * 32 + i + 1]);
+                            const float p2 = __uint_as_float(sr[c * 32 + i + 2]), p3 = __uint_as_float(sr[c * 32 + i + 3]);
                             l2a = fadd2(l2a, pack2(p0, p1));
                             l2b = fadd2(l2b, pack2(p2, p3));
                             __nv_bfloat162 pa = __floats2bfloat162_rn(p0, p1), pb = __floats2bfloat162_rn(p2, p3);
@@ -634,7 +655,10 @@ block_prefill_tc_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_c
             if (!ok) break;
             tc_fence_after();
             const float inv = l > 0.f ? 1.f / l : 0.f;
-            bf16* orow = reinterpret_cast<bf16*>(p.out) + ((size_t)it.bh * p.T + grow) * HD;
+            // O row -> bf16 -> the shared-memory stage that held this tile's last V tile (every MMA that
+            // read it is done), in the 128-byte-swizzled box layout, then one TMA store per box; rows
+            // past T are dropped by the store.  The stage goes back to the producer once read.
+            const uint32_t stage = sV + stage_o * TILE_BYTES + row * 128;
 #pragma unroll 1
             for (int c0 = 0; c0 < HD; c0 += 64) {
                 uint32_t o[64];
@@ -643,20 +667,30 @@ block_prefill_tc_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_c
                 tmem_wait_ld();
                 tmem_ld_fence32(o);
                 tmem_ld_fence32(o + 32);
-                if (grow < p.T) {
 #pragma unroll
-                    for (int q8 = 0; q8 < 8; ++q8) {
-                        float f[8];
+                for (int q8 = 0; q8 < 8; ++q8) {
+                    float f[8];
 #pragma unroll
-                        for (int i = 0; i < 8; ++i) f[i] = __uint_as_float(o[q8 * 8 + i]) * inv;
-                        *reinterpret_cast<uint4*>(orow + c0 + q8 * 8) = pack8(f);
-                    }
+                    for (int i = 0; i < 8; ++i) f[i] = __uint_as_float(o[q8 * 8 + i]) * inv;
+                    const uint4 w = pack8(f);
+                    const uint32_t dst = stage + (c0 >> 6) * kBoxBytes + ((q8 ^ (row & 7)) << 4);
+                    asm volatile("st.shared.v4.b32 [%0], {%1, %2, %3, %4};" ::"r"(dst), "r"(w.x), "r"(w.y), "r"(w.z), "r"(w.w) : "memory");
                 }
             }
-            // the next item's first P V overwrites O: it is issued only after this thread's next
-            // arrival on PFULL, which follows these loads in program order
             tc_fence_before();
+            asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+            asm volatile("barrier.sync.aligned %0, 128;" ::"r"(1 + x) : "memory");  // the warpgroup's 128 rows are staged
+            if (wq == 0 && lane == 0) {
+                for (int bx = 0; bx < NB; ++bx)
+                    tma_store_3d(&mapO, sV + stage_o * TILE_BYTES + bx * kBoxBytes, bx * 64, qt * BM, it.bh);
+                asm volatile("cp.async.bulk.commit_group;" ::: "memory");
+                asm volatile("cp.async.bulk.wait_group.read 0;" ::: "memory");
+                mbar_arrive(bar(B_VEMPTY + stage_o));
+            }
+            // the next item's first P V overwrites O: it is issued only after this thread's next
+            // arrival on P0FULL, which follows these loads in program order
         }
+        asm volatile("cp.async.bulk.wait_group 0;" ::: "memory");  // this thread's stores have landed
     }
 
     tc_fence_before();
@@ -730,12 +764,11 @@ static cudaError_t launch_t(const PrefillArgs& a, uint32_t* dev_status, cudaStre
         sm_count[dev] = n > 0 ? n : 1;
     }
     const long long slabs = (long long)a.B * a.H;
-    CUtensorMap mq, mk, mv;
+    CUtensorMap mq, mk, mv, mo;
     if (!make_map(&mq, a.q, HD, a.T, a.T, slabs) || !make_map(&mk, a.k, HD, a.T, a.kv_seq_stride, slabs) ||
-        !make_map(&mv, a.v, HD, a.T, a.kv_seq_stride, slabs))
+        !make_map(&mv, a.v, HD, a.T, a.kv_seq_stride, slabs) || !make_map(&mo, a.out, HD, a.T, a.T, slabs))
         return cudaErrorInvalidValue;
     Params p;
-    p.out = a.out;
     p.dev_status = dev_status;
     p.T = a.T;
     p.n_qtiles = (a.T + BM - 1) / BM;
@@ -746,7 +779,7 @@ static cudaError_t launch_t(const PrefillArgs& a, uint32_t* dev_status, cudaStre
     // cycle through all classes (heavy and light items alike)
     long long grid = p.n_items < sm_count[dev] ? p.n_items : sm_count[dev];
     while (grid > 1 && p.n_items > grid && gcd_int((int)grid, p.n_classes) != 1) --grid;
-    block_prefill_tc_kernel<HD><<<(unsigned)grid, kThreads, smem_bytes<HD>(), stream>>>(mq, mk, mv, p);
+    block_prefill_tc_kernel<HD><<<(unsigned)grid, kThreads, smem_bytes<HD>(), stream>>>(mq, mk, mv, mo, p);
     return cudaGetLastError();
 }
 
