@@ -108,43 +108,6 @@ __device__ __forceinline__ void attend_range(const bf16* __restrict__ qrow, cons
     }
 }
 
-// grid: B*H*splits CTAs.  splits == 1 writes bf16 output directly; otherwise each CTA writes
-// its normalised partial (hd floats) and its log2-sum-exp to the workspace.
-template <int HD>
-__global__ void __launch_bounds__(kDecodeThreads) block_decode_kernel(DecodeArgs a)
-{
-    constexpr int LPR = RowGeo<HD>::LPR;
-    __shared__ float smem[kDecodeWarps * (HD + 2)];
-    const int bh = blockIdx.x / a.splits, sp = blockIdx.x - bh * a.splits;
-    const int b = bh / a.H;
-    int n = a.len[b];
-    n = n < 0 ? 0 : (n > a.n_max ? a.n_max : n);
-    const int per = (n + a.splits - 1) / a.splits;
-    const int r0 = min(n, sp * per), r1 = min(n, r0 + per);
-
-    const bf16* Kb = reinterpret_cast<const bf16*>(a.k) + (size_t)bh * a.n_max * HD;
-    const bf16* Vb = reinterpret_cast<const bf16*>(a.v) + (size_t)bh * a.n_max * HD;
-    SoftmaxState st;
-    attend_range<HD>(reinterpret_cast<const bf16*>(a.q) + (size_t)bh * HD, Kb, Vb, r0, r1, a.scale_log2, st, smem);
-
-    if (threadIdx.x < LPR) {
-        const int sub = threadIdx.x;
-        float o[8];
-        float inv = st.l > 0.f ? 1.f / st.l : 0.f;
-#pragma unroll
-        for (int i = 0; i < 8; ++i) o[i] = st.acc[i] * inv;
-        if (a.splits == 1) {
-            *reinterpret_cast<uint4*>(reinterpret_cast<bf16*>(a.out) + (size_t)bh * HD + sub * 8) = pack8(o);
-        } else {
-            float* w = a.ws + ((size_t)bh * a.splits + sp) * kPartStride<HD>;
-            *reinterpret_cast<float4*>(w + sub * 8) = make_float4(o[0], o[1], o[2], o[3]);
-            *reinterpret_cast<float4*>(w + sub * 8 + 4) = make_float4(o[4], o[5], o[6], o[7]);
-            if (sub == 0) w[HD] = st.l > 0.f ? st.m + log2f(st.l) : kNegInf;
-        }
-        if (sub == 0 && sp == 0 && n == 0 && (bh % a.H) == 0) raise_status(a.dev_status, BT_DEV_EMPTY);
-    }
-}
-
 // Combine the per-split partials: out = sum_s w_s o_s with w_s = 2^(lse_s - max) / sum.
 // One lane group of LPR threads per (b,h).
 template <int HD>
@@ -179,8 +142,7 @@ template <int HD>
 static cudaError_t launch_decode_t(const DecodeArgs& a, cudaStream_t stream)
 {
     const int bh = a.B * a.H;
-    block_decode_kernel<HD><<<bh * a.splits, kDecodeThreads, 0, stream>>>(a);
-    cudaError_t e = cudaGetLastError();
+    cudaError_t e = launch_block_decode_ring(a, stream);
     if (e != cudaSuccess || a.splits == 1) return e;
     constexpr int LPR = RowGeo<HD>::LPR;
     const int groups_per_cta = 128 / LPR;

@@ -1,0 +1,313 @@
+// Block-decoder decode attention (paper section 2.3; appendix E.2), streaming form: the kernel
+// is bound by how many bytes of K and V it keeps in flight, so the bytes are moved by the bulk-copy
+// engine into shared-memory rings and the warps only compute.
+//
+// One persistent CTA per SM, eight warps.  Every warp works alone: it owns a ring of three 8 KB
+// stages (one stage = a chunk of K rows and the same rows of V), takes whole work items
+// ((sequence, head) or (sequence, head, split)), and lane 0 keeps two chunks in flight with
+// cp.async.bulk while the warp consumes the third - across item boundaries, so the stream never
+// drains.  No CTA-wide synchronisation exists; a stage is handed back by __syncwarp.  Per chunk a
+// lane group of hd/8 lanes owns a row: 128-bit shared-memory reads, fp32 dot product reduced by
+// shuffles, online softmax in the log2 domain per lane; row groups merge by shuffles at the end of
+// the item.  Every wait on a copy is bounded and raises BT_DEV_TIMEOUT when it runs out.
+#include "bt_common.cuh"
+#include "bt_kernels.h"
+
+namespace bt {
+namespace ring {
+
+#ifndef BT_DEC_WARPS
+#define BT_DEC_WARPS 8
+#endif
+#ifndef BT_DEC_STAGES
+#define BT_DEC_STAGES 3
+#endif
+#ifndef BT_DEC_UNROLL
+#define BT_DEC_UNROLL 8
+#endif
+constexpr int kWarps = BT_DEC_WARPS;
+constexpr int kThreads = kWarps * 32;
+constexpr int kStages = BT_DEC_STAGES;
+constexpr int kUnroll = BT_DEC_UNROLL;     // rows per lane group per chunk
+constexpr uint32_t kPollLimit = 1u << 24;  // polls of one wait before giving up (each poll suspends briefly)
+
+template <int HD>
+struct Geo {
+    static constexpr int LPR = RowGeo<HD>::LPR, RPW = RowGeo<HD>::RPW;
+    static constexpr int ROWS = kUnroll * RPW;          // rows per chunk: 32 at hd 64, 16 at hd 128
+    static constexpr int ROW_BYTES = HD * 2;
+    static constexpr int CHUNK_BYTES = ROWS * ROW_BYTES;  // 4096
+    static constexpr int STAGE_BYTES = 2 * CHUNK_BYTES;   // K chunk, then V chunk
+};
+template <int HD>
+constexpr int smem_bytes() { return kWarps * kStages * Geo<HD>::STAGE_BYTES + kWarps * kStages * 8; }
+
+__device__ __forceinline__ uint32_t smem_u32(const void* p) { return (uint32_t)__cvta_generic_to_shared(p); }
+
+__device__ __forceinline__ bool mbar_try_wait(uint32_t bar, uint32_t parity)
+{
+    uint32_t ok;
+    asm volatile(
+        "{\n\t.reg .pred p;\n\t"
+        "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
+        "selp.u32 %0, 1, 0, p;\n\t}"
+        : "=r"(ok)
+        : "r"(bar), "r"(parity)
+        : "memory");
+    return ok != 0;
+}
+__device__ __forceinline__ bool mbar_wait_bounded(uint32_t bar, uint32_t parity)
+{
+    for (uint32_t it = 0; it < kPollLimit; ++it)
+        if (mbar_try_wait(bar, parity)) return true;
+    return false;
+}
+// bytes global -> shared, completion counted on the mbarrier; the rows are read once, so they are
+// marked evict-first in L2
+__device__ __forceinline__ void bulk_load(uint32_t dst, const void* src, uint32_t bytes, uint32_t bar, uint64_t policy)
+{
+    asm volatile(
+        "cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes.L2::cache_hint [%0], [%1], %2, [%3], %4;"
+        ::"r"(dst), "l"(src), "r"(bytes), "r"(bar), "l"(policy)
+        : "memory");
+}
+__device__ __forceinline__ uint4 lds128(uint32_t addr)
+{
+    uint4 r;
+    asm volatile("ld.shared.v4.u32 {%0,%1,%2,%3}, [%4];" : "=r"(r.x), "=r"(r.y), "=r"(r.z), "=r"(r.w) : "r"(addr));
+    return r;
+}
+
+// Row range of one work item.
+struct Work {
+    int bh, sp, b, n, r0, r1;
+};
+__device__ __forceinline__ Work decode_work(int item, const DecodeArgs& a)
+{
+    Work w;
+    w.bh = item / a.splits;
+    w.sp = item - w.bh * a.splits;
+    w.b = w.bh / a.H;
+    int n = a.len[w.b];
+    n = n < 0 ? 0 : (n > a.n_max ? a.n_max : n);
+    w.n = n;
+    const int per = (n + a.splits - 1) / a.splits;
+    w.r0 = min(n, w.sp * per);
+    w.r1 = min(n, w.r0 + per);
+    return w;
+}
+
+// grid: one CTA per SM (fewer when there are fewer items than warps).  splits == 1 writes bf16
+// output directly; otherwise each item writes its normalised partial (hd floats) and its
+// log2-sum-exp to the workspace and decode_merge_kernel combines them.
+template <int HD>
+__global__ void __launch_bounds__(kThreads, 1) block_decode_ring_kernel(DecodeArgs a)
+{
+    using G = Geo<HD>;
+    constexpr int LPR = G::LPR, RPW = G::RPW, ROWS = G::ROWS;
+    extern __shared__ __align__(128) uint8_t smem[];
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    const int sub = lane % LPR, rg = lane / LPR;
+    const uint32_t ring0 = smem_u32(smem) + warp * (kStages * G::STAGE_BYTES);
+    const uint32_t bar0 = smem_u32(smem) + kWarps * kStages * G::STAGE_BYTES + warp * (kStages * 8);
+
+    if (lane == 0) {
+        for (int s = 0; s < kStages; ++s)
+            asm volatile("mbarrier.init.shared::cta.b64 [%0], 1;" ::"r"(bar0 + 8 * s) : "memory");
+        asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+    }
+    __syncwarp();
+    uint64_t policy;
+    asm volatile("createpolicy.fractional.L2::evict_first.b64 %0, 1.0;" : "=l"(policy));
+
+    const int n_items = a.B * a.H * a.splits;
+    const int stride = kWarps * gridDim.x;
+    const int first = warp * gridDim.x + blockIdx.x;   // neighbouring items go to different SMs
+    const bf16* Kall = reinterpret_cast<const bf16*>(a.k);
+    const bf16* Vall = reinterpret_cast<const bf16*>(a.v);
+
+    // ---- producer cursor (kept by every lane, acted on by lane 0): next chunk to request
+    int p_item = first, p_c = 0, p_nchunks = 0;
+    Work pw = {};
+    auto p_seek = [&]() {  // move to the next item that has rows
+        while (p_item < n_items) {
+            pw = decode_work(p_item, a);
+            p_nchunks = (pw.r1 - pw.r0 + ROWS - 1) / ROWS;
+            if (p_nchunks > 0) {
+                p_c = 0;
+                return;
+            }
+            p_item += stride;
+        }
+    };
+    uint32_t issued = 0, consumed = 0;
+    auto issue_one = [&]() {
+        if (p_item >= n_items) return;
+        const int row = pw.r0 + p_c * ROWS;
+        const uint32_t bytes = (uint32_t)min(ROWS, pw.r1 - row) * G::ROW_BYTES;
+        const uint32_t st = issued % kStages;
+        if (lane == 0) {
+            const uint32_t bar = bar0 + 8 * st, dst = ring0 + st * G::STAGE_BYTES;
+            const size_t off = ((size_t)pw.bh * a.n_max + row) * HD;
+            asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(bar), "r"(2 * bytes) : "memory");
+            bulk_load(dst, Kall + off, bytes, bar, policy);
+            bulk_load(dst + G::CHUNK_BYTES, Vall + off, bytes, bar, policy);
+        }
+        ++issued;
+        if (++p_c == p_nchunks) {
+            p_item += stride;
+            p_seek();
+        }
+    };
+    p_seek();
+    for (int s = 0; s < kStages; ++s) issue_one();
+
+    // ---- consumer: whole items, chunk by chunk
+    bool alive = true;
+    const bf16* Qall = reinterpret_cast<const bf16*>(a.q);
+    uint4 q_next = make_uint4(0, 0, 0, 0);  // the query of the next item is fetched an item ahead
+    if (first < n_items) q_next = ld_plain(Qall + (size_t)(first / a.splits) * HD + sub * 8);
+    for (int item = first; alive && item < n_items; item += stride) {
+        const Work w = decode_work(item, a);
+        float qf[8];
+        {
+            const uint4 qr = q_next;
+            if (item + stride < n_items) q_next = ld_plain(Qall + (size_t)((item + stride) / a.splits) * HD + sub * 8);
+            unpack8(qr, qf);
+#pragma unroll
+            for (int i = 0; i < 8; ++i) qf[i] *= a.scale_log2;
+        }
+        SoftmaxState st;
+        st.init();
+        const int nchunks = (w.r1 - w.r0 + ROWS - 1) / ROWS;
+        for (int c = 0; c < nchunks; ++c) {
+            const uint32_t sidx = consumed % kStages;
+            if (!mbar_wait_bounded(bar0 + 8 * sidx, (consumed / kStages) & 1)) {
+                alive = false;
+                break;
+            }
+            const int nvalid = min(ROWS, w.r1 - (w.r0 + c * ROWS));
+            const uint32_t ks = ring0 + sidx * G::STAGE_BYTES + rg * G::ROW_BYTES + sub * 16;
+            const uint32_t vs = ks + G::CHUNK_BYTES;
+            uint4 kr[kUnroll], vr[kUnroll];
+            float s[kUnroll];
+            float mt = kNegInf;
+            auto refill = [&]() {
+                ++consumed;
+                // the loaded values must be in registers, not merely requested, before the stage is overwritten
+#pragma unroll
+                for (int u = 0; u < kUnroll; ++u) asm volatile("" ::"r"(kr[u].x), "r"(vr[u].x) : "memory");
+                __syncwarp();
+                issue_one();
+            };
+            if (nvalid == ROWS) {
+#pragma unroll
+                for (int u = 0; u < kUnroll; ++u) kr[u] = lds128(ks + u * RPW * G::ROW_BYTES);
+#pragma unroll
+                for (int u = 0; u < kUnroll; ++u) vr[u] = lds128(vs + u * RPW * G::ROW_BYTES);
+                refill();   // the rows are in registers: request the next chunk before the arithmetic
+#pragma unroll
+                for (int u = 0; u < kUnroll; ++u) {
+                    s[u] = row_sum<LPR>(dot8(qf, kr[u]));
+                    mt = fmaxf(mt, s[u]);
+                }
+            } else {  // ragged tail: rows past the range were not copied and count as absent
+                const uint4 zero = make_uint4(0, 0, 0, 0);
+#pragma unroll
+                for (int u = 0; u < kUnroll; ++u) {
+                    const bool valid = u * RPW + rg < nvalid;
+                    kr[u] = valid ? lds128(ks + u * RPW * G::ROW_BYTES) : zero;
+                    vr[u] = valid ? lds128(vs + u * RPW * G::ROW_BYTES) : zero;
+                }
+                refill();
+#pragma unroll
+                for (int u = 0; u < kUnroll; ++u) {
+                    const float d = row_sum<LPR>(dot8(qf, kr[u]));
+                    s[u] = (u * RPW + rg < nvalid) ? d : kNegInf;
+                    mt = fmaxf(mt, s[u]);
+                }
+            }
+            if (mt != kNegInf) {  // uniform within the LPR lanes of a row group
+                const float mn = fmaxf(st.m, mt);
+                const float cf = ex2(st.m - mn);
+                st.l *= cf;
+#pragma unroll
+                for (int i = 0; i < 8; ++i) st.acc[i] *= cf;
+#pragma unroll
+                for (int u = 0; u < kUnroll; ++u) {
+                    const float p = ex2(s[u] - mn);
+                    st.l += p;
+                    fma8(st.acc, p, vr[u]);
+                }
+                st.m = mn;
+            }
+        }
+        if (!alive) break;
+        // merge the RPW row groups of the warp
+#pragma unroll
+        for (int off = LPR; off < 32; off <<= 1) {
+            const float m2 = __shfl_xor_sync(0xffffffffu, st.m, off);
+            const float l2 = __shfl_xor_sync(0xffffffffu, st.l, off);
+            float a2[8];
+#pragma unroll
+            for (int i = 0; i < 8; ++i) a2[i] = __shfl_xor_sync(0xffffffffu, st.acc[i], off);
+            st.merge(m2, l2, a2);
+        }
+        if (rg == 0) {
+            float o[8];
+            const float inv = st.l > 0.f ? 1.f / st.l : 0.f;
+#pragma unroll
+            for (int i = 0; i < 8; ++i) o[i] = st.acc[i] * inv;
+            if (a.splits == 1) {
+                *reinterpret_cast<uint4*>(reinterpret_cast<bf16*>(a.out) + (size_t)w.bh * HD + sub * 8) = pack8(o);
+            } else {
+                float* ws = a.ws + ((size_t)w.bh * a.splits + w.sp) * (HD + 4);
+                *reinterpret_cast<float4*>(ws + sub * 8) = make_float4(o[0], o[1], o[2], o[3]);
+                *reinterpret_cast<float4*>(ws + sub * 8 + 4) = make_float4(o[4], o[5], o[6], o[7]);
+                if (sub == 0) ws[HD] = st.l > 0.f ? st.m + log2f(st.l) : kNegInf;
+            }
+            if (sub == 0 && w.sp == 0 && w.n == 0 && (w.bh % a.H) == 0) raise_status(a.dev_status, BT_DEV_EMPTY);
+        }
+    }
+    if (!alive) {
+        // a copy never completed: report it, give the copies still in flight one more bounded wait so
+        // that none lands in shared memory after the CTA is gone, and leave
+        if (lane == 0) raise_status(a.dev_status, BT_DEV_TIMEOUT);
+        for (; consumed < issued; ++consumed)
+            if (!mbar_wait_bounded(bar0 + 8 * (consumed % kStages), (consumed / kStages) & 1)) break;
+    }
+}
+
+template <int HD>
+static cudaError_t launch_t(const DecodeArgs& a, cudaStream_t stream)
+{
+    constexpr int kMaxDevices = 64;
+    static int sm_count[kMaxDevices];  // 0 = this device has not been set up yet
+    int dev = 0;
+    cudaError_t e = cudaGetDevice(&dev);
+    if (e != cudaSuccess) return e;
+    if (dev < 0 || dev >= kMaxDevices) return cudaErrorInvalidDevice;
+    if (!sm_count[dev]) {
+        e = cudaFuncSetAttribute(block_decode_ring_kernel<HD>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem_bytes<HD>());
+        if (e != cudaSuccess) return e;
+        int n = 0;
+        e = cudaDeviceGetAttribute(&n, cudaDevAttrMultiProcessorCount, dev);
+        if (e != cudaSuccess) return e;
+        sm_count[dev] = n > 0 ? n : 1;
+    }
+    const long long items = (long long)a.B * a.H * a.splits;
+    if (items > 0x7fffffffLL - 4096) return cudaErrorInvalidConfiguration;
+    // one CTA per SM; with few items, one item per CTA first so that they spread over the SMs
+    long long grid = items < sm_count[dev] ? items : sm_count[dev];
+    block_decode_ring_kernel<HD><<<(unsigned)grid, kThreads, smem_bytes<HD>(), stream>>>(a);
+    return cudaGetLastError();
+}
+
+}  // namespace ring
+
+cudaError_t launch_block_decode_ring(const DecodeArgs& a, cudaStream_t stream)
+{
+    return a.hd == 64 ? ring::launch_t<64>(a, stream) : ring::launch_t<128>(a, stream);
+}
+
+}  // namespace bt

@@ -34,6 +34,8 @@ struct DecodeArgs {
     float scale_log2;    // softmax scale * log2(e)
 };
 cudaError_t launch_block_decode(const DecodeArgs& a, cudaStream_t stream);
+// The streaming kernel alone (per-item results or per-split partials; no merge pass).
+cudaError_t launch_block_decode_ring(const DecodeArgs& a, cudaStream_t stream);
 
 struct TokenArgs {
     void* kv;            // layer base, [B][H][C][2][hd]
