@@ -55,6 +55,39 @@ class BlockDecodeStep:
                 e1.record()
                 attn_events.append((e0, e1))
 
+    def _capture(self, events):
+        g = torch.cuda.CUDAGraph()
+        with torch.cuda.graph(g):
+            self.rewind()
+            for l in range(self.w.n_layers):
+                bt.bt_block_kv_append(self.cfg, self.cache, l, self.k_new[l], self.v_new[l], n_new=1, dev_status=self.status)
+                if events is not None:
+                    e0 = torch.cuda.Event(enable_timing=True, external=True)
+                    e1 = torch.cuda.Event(enable_timing=True, external=True)
+                    e0.record()
+                bt.bt_block_decode_attn(self.cfg, self.cache, l, self.q[l], self.out[l], self.ws, dev_status=self.status)
+                if events is not None:
+                    e1.record()
+                    events.append((e0, e1))
+        return g
+
+    def capture(self):
+        """Capture rewind + one whole step into two CUDA graphs: a plain one (replay) and one with
+        timing events (external, so that they may sit inside a graph) around every attention launch
+        (replay_timed; after it the events hold that replay's per-launch times)."""
+        self.step()  # anything lazy (module load, per-device set-up) happens outside the capture
+        self.rewind()
+        torch.cuda.synchronize()
+        self.graph = self._capture(None)
+        self.graph_events = []
+        self.graph_timed = self._capture(self.graph_events)
+
+    def replay_timed(self):
+        self.graph_timed.replay()
+
+    def replay(self):
+        self.graph.replay()
+
     # ---- the same step driven from pinned host buffers through bt_block_decode_step_host
     def _host_buffers(self):
         if self._host is None:
@@ -91,14 +124,22 @@ class TokenDecodeRun:
         self.t = 0
         self.launches_per_step = w.n_layers
 
-    def token_step(self):
-        """Token step t (prefix length 1: the prefix row is the first row of each block)."""
+    def token_step(self, events=None):
+        """Token step t (prefix length 1: the prefix row is the first row of each block).  events: optional
+        list receiving an (external) timing event pair around every launch."""
         w = self.w
         j = self.t % w.block_len
         r = self.t % self.ring
         for l in range(w.n_layers):
+            if events is not None:
+                e0 = torch.cuda.Event(enable_timing=True, external=True)
+                e1 = torch.cuda.Event(enable_timing=True, external=True)
+                e0.record()
             bt.bt_token_decode_attn(self.cfg, self.cache, l, self.q[r, l], self.k_new[r, l], self.v_new[r, l], self.out[l],
                                     n_q=1, reset_first=(j == 0), dev_status=self.status)
+            if events is not None:
+                e1.record()
+                events.append((e0, e1))
         self.t += 1
 
     def capture(self, n_steps=None):

@@ -1,0 +1,95 @@
+"""GPU parity at the full workload sizes, in the launch configuration bench.py times (the harness
+drivers): the CUDA path runs the whole workload, the oracle recomputes sampled sequences from
+exactly the bytes the GPU used (copied back), and everything integer (lengths, appended rows) is
+checked bit-exactly over the full size."""
+import numpy as np
+import pytest
+import torch
+
+import oracle
+from oracle import schedule
+from workloads import configs, gen
+
+from util import assert_close, local_kv_split
+
+pytestmark = pytest.mark.gpu
+
+
+@pytest.fixture(scope="module")
+def bt():
+    import paper_2406_02657_b200 as bt
+    assert torch.cuda.is_available()
+    return bt
+
+
+def _fill(w):
+    return lambda tid, shape: gen.normal_bf16_device(w.seed, tid, shape, device="cuda")
+
+
+def test_block_decode_step_full_size(bt):
+    """BASELINE configs[1]: batch 256, 16 heads, head_dim 64, 512 rows after the append, 12 layers."""
+    from paper_2406_02657_b200 import harness
+    w = configs.BLOCK_DECODE
+    run = harness.BlockDecodeStep(w, fill=_fill(w))
+    k_before = {l: gen.torch_to_bits(run.cache.k[l, :, :, w.ctx_blocks - 1]) for l in (0, 5)}  # the row the append overwrites
+    run.step()
+    torch.cuda.synchronize()
+    assert run.status.item() == 0
+    assert (run.cache.len == w.ctx_blocks).all()  # every (layer, sequence) advanced by exactly one row
+    # the appended rows are the new rows, bit for bit, over the whole batch
+    for l in range(w.n_layers):
+        assert torch.equal(run.cache.k[l, :, :, w.ctx_blocks - 1], run.k_new[l, :, :, 0])
+        assert torch.equal(run.cache.v[l, :, :, w.ctx_blocks - 1], run.v_new[l, :, :, 0])
+    assert not np.array_equal(k_before[0], gen.torch_to_bits(run.k_new[0, :, :, 0]))  # the check above is not vacuous
+    # sampled sequences, every head, first / middle / last layer: outputs against the oracle
+    seqs = [0, 1, 97, 128, 254, 255]
+    for l in (0, 5, w.n_layers - 1):
+        c = oracle.Cache(len(seqs), w.heads, w.max_blocks, w.head_dim)
+        c.k[...] = gen.torch_to_bits(run.cache.k[l][seqs])
+        c.v[...] = gen.torch_to_bits(run.cache.v[l][seqs])
+        c.len[...] = w.ctx_blocks
+        ref = oracle.block_decode_attn(c, gen.torch_to_bits(run.q[l][seqs][:, :, 0]))
+        assert_close(run.out[l][seqs][:, :, 0], ref, f"full-size block decode layer {l}")
+
+
+def test_token_decode_full_size_two_blocks(bt):
+    """BASELINE configs[2]: 4096 sequences, 12 layers, local cache 1 prefix + up to L_B rows; two
+    blocks of consecutive token steps, lengths against the integer schedule model at full size."""
+    from paper_2406_02657_b200 import harness
+    w = configs.TOKEN_DECODE
+    run = harness.TokenDecodeRun(w, fill=_fill(w))
+    seqs = [0, 5, 2047, 4095]
+    layers = (0, w.n_layers - 1)
+    ocache = {l: oracle.Cache(len(seqs), w.heads, w.local_cap, w.head_dim) for l in layers}
+    n_steps = 2 * w.block_len
+    sched = schedule.token_step_schedule(w.block_len, w.prefix_len, n_steps)
+    for t in range(n_steps):
+        r = t % run.ring
+        run.token_step()
+        torch.cuda.synchronize()
+        reset, n_app, len_after = sched[t]
+        assert (run.cache.len == len_after).all(), f"step {t}: lengths differ from the schedule model"
+        for l in layers:
+            q, k, v = (gen.torch_to_bits(x[r, l][seqs]) for x in (run.q, run.k_new, run.v_new))
+            ref = oracle.token_decode_attn(ocache[l], q, k, v, reset_first=bool(reset))
+            assert_close(run.out[l][seqs], ref, f"full-size token step {t} layer {l}")
+            assert np.array_equal(ocache[l].len, np.full(len(seqs), len_after, np.int32))
+            gk, gv = local_kv_split(run.cache.kv[l][seqs])
+            n = len_after
+            assert np.array_equal(gk[:, :, :n], ocache[l].k[:, :, :n]) and np.array_equal(gv[:, :, :n], ocache[l].v[:, :, :n])
+    assert run.status.item() == 0
+
+
+def test_block_prefill_full_size(bt):
+    """BASELINE configs[3]: batch 32, 512 prompt blocks, 16 heads, head_dim 128, 12 layers."""
+    from paper_2406_02657_b200 import harness
+    w = configs.BLOCK_PREFILL
+    run = harness.PrefillRun(w, fill=_fill(w))
+    run.out.fill_(float("nan"))
+    run.step()
+    torch.cuda.synchronize()
+    assert torch.isfinite(run.out.float()).all()  # every row of every layer was written
+    for l, b, h in ((0, 0, 0), (0, 31, 15), (6, 13, 7), (11, 31, 0), (11, 5, 15)):
+        q, k, v = (gen.torch_to_bits(x[l, b:b + 1, h:h + 1]) for x in (run.q, run.k, run.v))
+        ref = oracle.block_prefill_attn(q, k, v)
+        assert_close(run.out[l, b:b + 1, h:h + 1], ref, f"full-size prefill layer {l} b {b} h {h}", p_bf16=True)
