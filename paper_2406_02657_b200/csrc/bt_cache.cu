@@ -17,6 +17,10 @@ __global__ void __launch_bounds__(kAppendThreads) kv_append_kernel(CacheView c, 
                                                                    uint32_t* dev_status)
 {
     const int b = blockIdx.x;
+    if (kFused) {  // launched with launch_pdl
+        pdl_launch_dependents();
+        pdl_wait();
+    }
     const int len = c.len[b];
     if (kFused) __syncthreads();
     const bool ok = len >= 0 && len + n_new <= c.cap;
@@ -70,8 +74,7 @@ cudaError_t launch_kv_append(const CacheView& c, int B, int H, int hd, const voi
     const bf16* kn = reinterpret_cast<const bf16*>(k_new);
     const bf16* vn = reinterpret_cast<const bf16*>(v_new);
     if (chunks <= 4 * kAppendThreads) {
-        kv_append_kernel<true><<<dim3(B, 1), kAppendThreads, 0, stream>>>(c, H, hd, kn, vn, n_new, dev_status);
-        return cudaGetLastError();
+        return launch_pdl(kv_append_kernel<true>, dim3(B, 1), dim3(kAppendThreads), 0, stream, c, H, hd, kn, vn, n_new, dev_status);
     }
     long long gy = (chunks + 4 * kAppendThreads - 1) / (4 * kAppendThreads);
     if (gy > 1024) gy = 1024;

@@ -123,6 +123,30 @@ struct SoftmaxState {
     }
 };
 
+// Programmatic dependent launch.  A kernel launched with launch_pdl may start while the kernel
+// before it in the stream is still draining: it calls pdl_launch_dependents() first (its own
+// successor may then be scheduled as soon as SM resources free up) and pdl_wait() before its first
+// access to global memory - the wait returns once the preceding kernel has completed and its
+// writes are visible, so the kernel sees exactly what ordinary stream order would show it.
+__device__ __forceinline__ void pdl_launch_dependents() { asm volatile("griddepcontrol.launch_dependents;" ::: "memory"); }
+__device__ __forceinline__ void pdl_wait() { asm volatile("griddepcontrol.wait;" ::: "memory"); }
+
+template <typename... KArgs, typename... Args>
+inline cudaError_t launch_pdl(void (*kernel)(KArgs...), dim3 grid, dim3 block, size_t smem, cudaStream_t stream, Args&&... args)
+{
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = grid;
+    cfg.blockDim = block;
+    cfg.dynamicSmemBytes = smem;
+    cfg.stream = stream;
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr[0].val.programmaticStreamSerializationAllowed = 1;
+    cfg.attrs = attr;
+    cfg.numAttrs = 1;
+    return cudaLaunchKernelEx(&cfg, kernel, KArgs(args)...);
+}
+
 __device__ __forceinline__ void raise_status(uint32_t* dev_status, uint32_t bits)
 {
     if (dev_status && bits) atomicOr(dev_status, bits);

@@ -119,6 +119,8 @@ __global__ void __launch_bounds__(kThreads, 1) block_decode_ring_kernel(DecodeAr
     __syncwarp();
     uint64_t policy;
     asm volatile("createpolicy.fractional.L2::evict_first.b64 %0, 1.0;" : "=l"(policy));
+    pdl_launch_dependents();
+    pdl_wait();  // nothing above touched global memory
 
     const int n_items = a.B * a.H * a.splits;
     const int stride = kWarps * gridDim.x;
@@ -299,8 +301,7 @@ static cudaError_t launch_t(const DecodeArgs& a, cudaStream_t stream)
     if (items > 0x7fffffffLL - 4096) return cudaErrorInvalidConfiguration;
     // one CTA per SM; with few items, one item per CTA first so that they spread over the SMs
     long long grid = items < sm_count[dev] ? items : sm_count[dev];
-    block_decode_ring_kernel<HD><<<(unsigned)grid, kThreads, smem_bytes<HD>(), stream>>>(a);
-    return cudaGetLastError();
+    return launch_pdl(block_decode_ring_kernel<HD>, dim3((unsigned)grid), dim3(kThreads), (size_t)smem_bytes<HD>(), stream, a);
 }
 
 }  // namespace ring

@@ -217,6 +217,8 @@ token_step_pipelined_kernel(TokenArgs a, int seqs_per_cta, int threads_per_seq)
     // kLenAhead groups before that.
     constexpr int kLenAhead = 3, kLens = kDepth + kLenAhead;
     int lens[kLens];
+    pdl_launch_dependents();
+    pdl_wait();  // nothing above touched global memory
 #pragma unroll
     for (int d = 0; d < kLens; ++d) lens[d] = load_len(seq_of(d));
 #pragma unroll
@@ -338,8 +340,8 @@ static cudaError_t launch_pipelined(const TokenArgs& a, int spc, int tps, cudaSt
     const int n_groups = (a.B + spc - 1) / spc;
     const int slots = sm_count() * kCtasPerSm;
     const int grid = n_groups < slots ? n_groups : slots;
-    token_step_pipelined_kernel<HD, kDepth, kMaxRows, kCtasPerSm><<<grid, kTokThreads, smem, stream>>>(a, spc, tps);
-    return cudaGetLastError();
+    return launch_pdl(token_step_pipelined_kernel<HD, kDepth, kMaxRows, kCtasPerSm>, dim3(grid), dim3(kTokThreads), smem, stream,
+                      a, spc, tps);
 }
 
 cudaError_t launch_token_decode(const TokenArgs& a, cudaStream_t stream)
