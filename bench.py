@@ -155,10 +155,10 @@ def run_reference(args):
     if rank != 0:
         return 0
     import oracle
-    w = configs.BY_NAME[args.workload]
     if args.workload != "block_decode":
         print(json.dumps({"impl": "reference", "unavailable": "reference arm implemented for the block_decode workload only"}))
         return 0
+    w = configs.BY_NAME[args.workload]
     n_seq = 64
     for _ in range(max(1, min(args.warmup, 2))):
         oracle_block_decode_sample(w, n_seq)
@@ -191,6 +191,11 @@ def workload_config(w, name):
     elif name == "token_decode":
         c.update(workload="token_decode: BASELINE configs[2], fused reset+append+local attention, 12 launches per token step",
                  l2="no flush: inputs rotate over a ring larger than L2")
+    elif name == "sweep":
+        c.update(workload=f"sweep: BASELINE configs[4], decode-heavy generation at L_B = {w.block_len}: prompt {w.prompt_tokens} tokens, "
+                          f"{w.gen_tokens} generated, block step every L_B tokens and token step every token",
+                 prompt_tokens=w.prompt_tokens, gen_tokens=w.gen_tokens, max_blocks=w.max_blocks,
+                 l2="no flush: the block cache alone is far larger than L2")
     elif name == "block_prefill":
         c.update(workload="block_prefill: BASELINE configs[3], dense causal attention over 512 prompt blocks",
                  prompt_blocks=w.prompt_blocks, l2="no flush: 3.2 GB of Q,K,V,out per step")
@@ -212,7 +217,7 @@ def run_gpu(args):
     import paper_2406_02657_b200 as bt  # noqa: F401  (loads libbt.so; raises if it cannot)
     from paper_2406_02657_b200 import harness
 
-    w = configs.BY_NAME[args.workload]
+    w = configs.sweep(args.block_len) if args.workload == "sweep" else configs.BY_NAME[args.workload]
     reduced = {}
     if args.batch:
         reduced["batch"] = args.batch
@@ -288,6 +293,24 @@ def run_gpu(args):
         dom = "token_decode_kernel"
         launches = run.launches_per_step * n_tok * args.steps
         step_bytes = w.n_layers * alg_bytes
+    elif args.workload == "sweep":
+        # a bench step = one whole generation: prompt prefill + bulk append, then gen_tokens / L_B generated
+        # blocks (CUDA-graph replays of `ring` blocks each); tokens = batch x generated tokens
+        run = harness.GenerationRun(w, fill=fill)
+        run.capture()
+        tokens_per_step = w.batch * w.gen_tokens
+        sampler.start()
+        ms = timed(run.generate, lambda: None, args.steps, args.warmup)
+        clocks = sampler.stop()
+        assert run.status.item() == 0 and (run.block.len == w.max_blocks).all()
+        ms_e2e, h2d, d2h = None, 0, 0
+        parts = traffic.generation_bytes(w.batch, w.heads, w.head_dim, w.n_layers, w.block_len, w.prompt_tokens, w.gen_tokens)
+        step_bytes = parts["total"]
+        n_blocks = w.gen_tokens // w.block_len
+        launches = (run.launches_prefill + run.launches_per_block * n_blocks) * args.steps
+        dom = "block_decode_ring_kernel (whole generation: all kernels)"
+        alg_bytes = step_bytes
+        run.launches_per_step = 1  # the roofline line below is for the whole generation
     else:
         run = harness.PrefillRun(w, fill=fill)
         tokens_per_step = w.batch * w.prompt_tokens
@@ -344,14 +367,17 @@ def run_gpu(args):
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
-    ap.add_argument("--steps", type=int, default=200)
+    ap.add_argument("--steps", type=int, default=0, help="timed steps (default 200; 3 for the sweep, whose step is a whole generation)")
     ap.add_argument("--warmup", type=int, default=3)
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
-    ap.add_argument("--workload", default="block_decode", choices=["block_decode", "token_decode", "block_prefill"])
+    ap.add_argument("--workload", default="block_decode", choices=["block_decode", "token_decode", "block_prefill", "sweep"])
+    ap.add_argument("--block-len", type=int, default=4, help="L_B of the generation sweep (1, 2, 4 or 8)")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--batch", type=int, default=0, help="override the batch (profiling a small case; not a bench number)")
     ap.add_argument("--layers", type=int, default=0, help="override the layer count (profiling a small case)")
     args = ap.parse_args()
+    if args.steps <= 0:
+        args.steps = 3 if args.workload == "sweep" else 200
     if args.warmup < 3 and args.impl == "ours":
         args.warmup = 3
     if args.impl == "reference":

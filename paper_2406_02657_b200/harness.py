@@ -183,3 +183,76 @@ class PrefillRun:
             if events is not None:
                 e1.record()
                 events.append((e0, e1))
+
+
+class GenerationRun:
+    """Decode-heavy generation (section 3.2: 128-token prompt, 2048 generated tokens) through both
+    decoders' attention: prefill of the prompt's T blocks and bulk append of their K,V rows, then per
+    generated block L_B token-decoder steps (reset at the first) and one block-decoder step (append
+    one row, attend over all rows), n_layers each.  Step inputs rotate over a small ring of
+    pre-drawn tensors; one pass over the ring is captured as a CUDA graph and replayed."""
+
+    def __init__(self, w, device="cuda", fill=None, ring=4):
+        self.w, self.device, self.ring = w, device, ring
+        L, B, H, hd = w.n_layers, w.batch, w.heads, w.head_dim
+        self.cfg = bt.make_config(B, H, hd, w.block_len, w.prefix_len, w.max_blocks, L)
+        mk = (lambda tid, shape: fill(tid, shape)) if fill is not None else \
+            (lambda tid, shape: torch.zeros(shape, dtype=torch.bfloat16, device=device))
+        T = w.prompt_blocks
+        self.pq, self.pk, self.pv = (mk(20 + i, (L, B, H, T, hd)) for i in range(3))
+        self.pout = torch.empty((L, B, H, T, hd), dtype=torch.bfloat16, device=device)
+        self.bq, self.bk, self.bv = (mk(23 + i, (ring, L, B, H, 1, hd)) for i in range(3))
+        self.bout = torch.empty((L, B, H, 1, hd), dtype=torch.bfloat16, device=device)
+        self.tq, self.tk, self.tv = (mk(26 + i, (ring, w.block_len, L, B, H, 1, hd)) for i in range(3))
+        self.tout = torch.empty((L, B, H, 1, hd), dtype=torch.bfloat16, device=device)
+        self.block = bt.BlockCache(self.cfg, device, k=torch.empty((L, B, H, w.max_blocks, hd), dtype=torch.bfloat16, device=device),
+                                   v=torch.empty((L, B, H, w.max_blocks, hd), dtype=torch.bfloat16, device=device))
+        self.local = bt.LocalCache(self.cfg, device)
+        self.ws = bt.alloc_workspace(self.cfg, device)
+        self.status = torch.zeros(1, dtype=torch.int32, device=device)
+        self.n_gen_blocks = w.gen_tokens // w.block_len
+        self.graph = None
+        self.launches_prefill = 2 * L
+        self.launches_per_block = L * (w.block_len + 2 + (1 if bt.bt_decode_splits(self.cfg) > 1 else 0))
+
+    def start(self):
+        """Empty caches, then the prompt: prefill attention and bulk append per layer."""
+        self.block.len.zero_()
+        self.local.len.zero_()
+        w = self.w
+        for l in range(w.n_layers):
+            bt.bt_block_prefill_attn(self.cfg, self.pq[l], self.pk[l], self.pv[l], self.pout[l], n_blocks=w.prompt_blocks,
+                                     dev_status=self.status)
+            bt.bt_block_kv_append(self.cfg, self.block, l, self.pk[l], self.pv[l], n_new=w.prompt_blocks, dev_status=self.status)
+
+    def gen_block(self, r):
+        """One generated block with ring slot r: L_B token steps, then the block step."""
+        w = self.w
+        for j in range(w.block_len):
+            for l in range(w.n_layers):
+                bt.bt_token_decode_attn(self.cfg, self.local, l, self.tq[r, j, l], self.tk[r, j, l], self.tv[r, j, l], self.tout[l],
+                                        n_q=1, reset_first=(j == 0), dev_status=self.status)
+        for l in range(w.n_layers):
+            bt.bt_block_kv_append(self.cfg, self.block, l, self.bk[r, l], self.bv[r, l], n_new=1, dev_status=self.status)
+            bt.bt_block_decode_attn(self.cfg, self.block, l, self.bq[r, l], self.bout[l], self.ws, dev_status=self.status)
+
+    def capture(self):
+        """One pass over the input ring (ring generated blocks) as a CUDA graph."""
+        assert self.n_gen_blocks % self.ring == 0
+        self.start()
+        self.gen_block(0)  # anything lazy happens outside the capture
+        torch.cuda.synchronize()
+        self.graph = torch.cuda.CUDAGraph()
+        with torch.cuda.graph(self.graph):
+            for r in range(self.ring):
+                self.gen_block(r)
+
+    def generate(self):
+        """The whole generation: prompt, then n_gen_blocks generated blocks (graph replays)."""
+        self.start()
+        if self.graph is None:
+            for g in range(self.n_gen_blocks):
+                self.gen_block(g % self.ring)
+        else:
+            for _ in range(self.n_gen_blocks // self.ring):
+                self.graph.replay()

@@ -41,3 +41,14 @@ def prefill_layer_flops(B: int, H: int, T: int, hd: int) -> int:
     """Causal attention: T(T+1)/2 (query, key) pairs, each 2*hd flops for the score and 2*hd
     for the weighted sum."""
     return B * H * (T * (T + 1) // 2) * 4 * hd
+
+
+def generation_bytes(B: int, H: int, hd: int, n_layers: int, block_len: int, prompt_tokens: int, gen_tokens: int) -> dict:
+    """Whole decode-heavy generation: prompt prefill + bulk append, then per generated block L_B token
+    steps (step j reads j cached rows) and one block step over T + g + 1 rows.  Returns the parts."""
+    T = prompt_tokens // block_len
+    G = gen_tokens // block_len
+    prefill = n_layers * (prefill_layer_bytes(B, H, T, hd) + 2 * 2 * B * H * T * hd * BF16)
+    token = n_layers * G * sum(token_decode_layer_bytes(B, H, hd, j) for j in range(block_len))
+    block = n_layers * sum(block_decode_layer_bytes(B, H, hd, T + g + 1, True) for g in range(G))
+    return {"prefill": prefill, "token": token, "block": block, "total": prefill + token + block}
