@@ -31,6 +31,17 @@ constexpr uint32_t kSpinLimit = 1u << 26;
 constexpr uint64_t kWaitLimitNs = 1000000000ull;  // 1 s: far beyond any legitimate wait
 constexpr float kRescaleThreshold = 8.0f;  // log2 units
 
+// Optional event timeline (compiled in only with -DBT_PF_TRACE; a development aid, off in the library):
+// CTA 0 records (clock, event id) pairs per role into p.trace[role][kTraceEvents].
+#ifdef BT_PF_TRACE
+constexpr int kTraceEvents = 4096;
+#define PF_EV_DECL int ev_n = 0
+#define PF_EV(role, id) do { if (p.trace && blockIdx.x == 0 && ev_n < kTraceEvents) { p.trace[(role) * kTraceEvents + ev_n] = (clock64() << 8) | (long long)(id); ++ev_n; } } while (0)
+#else
+#define PF_EV_DECL
+#define PF_EV(role, id)
+#endif
+
 __device__ __forceinline__ uint32_t smem_u32(const void* p) { return (uint32_t)__cvta_generic_to_shared(p); }
 
 __device__ __forceinline__ void mbar_init(uint32_t bar, uint32_t count)
@@ -57,6 +68,19 @@ __device__ __forceinline__ bool mbar_try_wait(uint32_t bar, uint32_t parity)
         : "memory");
     return ok != 0;
 }
+// Non-blocking test: much cheaper than try_wait when the phase has already completed.
+__device__ __forceinline__ bool mbar_test_wait(uint32_t bar, uint32_t parity)
+{
+    uint32_t ok;
+    asm volatile(
+        "{\n\t.reg .pred p;\n\t"
+        "mbarrier.test_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
+        "selp.u32 %0, 1, 0, p;\n\t}"
+        : "=r"(ok)
+        : "r"(bar), "r"(parity)
+        : "memory");
+    return ok != 0;
+}
 __device__ __forceinline__ uint64_t global_ns()
 {
     uint64_t t;
@@ -67,6 +91,7 @@ __device__ __forceinline__ uint64_t global_ns()
 // the limit ran out or another thread of the CTA gave up.
 __device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatile int* abort_flag, uint32_t* dev_status)
 {
+    if (mbar_test_wait(bar, parity)) return true;
     uint64_t t0 = 0;
     for (uint32_t it = 0; it < kSpinLimit; ++it) {
         if (mbar_try_wait(bar, parity)) return true;
@@ -300,7 +325,13 @@ struct Params {
     int T, n_qtiles, n_classes;
     long long n_items;
     float scale_log2;
+#ifdef BT_PF_TRACE
+    long long* trace;
+#endif
 };
+#ifdef BT_PF_TRACE
+long long* g_trace = nullptr;
+#endif
 
 // warps 0-3: softmax warpgroup of tile A, warps 4-7: of tile B
 constexpr int kProducerWarp = 8, kMmaWarp = 9;
@@ -447,21 +478,26 @@ block_prefill_tc_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_c
             uint32_t q_uses[kQBufs] = {0, 0, 0};
             uint32_t kv_base = 0;                 // key/value tiles consumed by earlier items
             uint32_t p_count[2] = {0, 0};         // P tiles consumed so far, per query tile slot
-            uint32_t n_done = 0;
             bool ok = true;
+            uint32_t n_done = 0;
+            PF_EV_DECL;
             for (long long item = blockIdx.x; ok && item < p.n_items; item += gridDim.x, ++n_done) {
                 const Item it = decode_item(item, p);
+                PF_EV(2, 20);
                 const int qbuf[2] = {(n_done & 1) ? 2 : 0, 1};
                 const int steps[2] = {it.na, it.nb};
                 // S_x(j) = Q_x K_j^T, then the barriers that fire when it (and all before it) is done
                 auto issue_s = [&](int x, int j) {
                     const uint32_t kc = kv_base + j, st = kc % kKvStages;
+                    PF_EV(2, 0 + 32 * x);
                     ok = ok && mbar_wait(bar(B_KFULL + st), (kc / kKvStages) & 1, abort_flag, p.dev_status);
+                    PF_EV(2, 1 + 32 * x);
                     if (ok && j == 0) {
                         ok = mbar_wait(bar(B_QFULL + qbuf[x]), q_uses[qbuf[x]] & 1, abort_flag, p.dev_status);
                         ++q_uses[qbuf[x]];
                     }
                     if (!ok) return;
+                    PF_EV(2, 2 + 32 * x);
                     tc_fence_after();
                     const uint32_t q0 = sQ + qbuf[x] * TILE_BYTES, k0 = sK + st * TILE_BYTES;
 #pragma unroll
@@ -474,12 +510,15 @@ block_prefill_tc_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_c
                     if (j == steps[x] - 1) mma_commit(bar(B_QEMPTY + qbuf[x]));  // last use of this Q tile
                     // K_j is free after its last reader: tile B while it still runs, else tile A
                     if (x == 1 || j >= it.nb) mma_commit(bar(B_KEMPTY + st));
+                    PF_EV(2, 3 + 32 * x);
                 };
                 // O_x (+)= P_x(j) V_j
                 auto issue_pv = [&](int x, int j) {
                     const uint32_t kc = kv_base + j, st = kc % kKvStages;
-                    ok = ok && mbar_wait(bar(B_P0FULL + x), p_count[x] & 1, abort_flag, p.dev_status) &&
-                         mbar_wait(bar(B_VFULL + st), (kc / kKvStages) & 1, abort_flag, p.dev_status);
+                    ok = ok && mbar_wait(bar(B_P0FULL + x), p_count[x] & 1, abort_flag, p.dev_status);
+                    PF_EV(2, 4 + 32 * x);
+                    ok = ok && mbar_wait(bar(B_VFULL + st), (kc / kKvStages) & 1, abort_flag, p.dev_status);
+                    PF_EV(2, 5 + 32 * x);
                     if (!ok) return;
                     tc_fence_after();
                     const uint32_t v0 = sV + st * TILE_BYTES;
@@ -493,7 +532,9 @@ block_prefill_tc_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_c
                     // the softmax warps still work on the last quarter
 #pragma unroll
                     for (int kk = 0; kk < kEarlyChunks * 2; ++kk) pv(kk);
+                    PF_EV(2, 6 + 32 * x);
                     ok = mbar_wait(bar(B_P1FULL + x), p_count[x] & 1, abort_flag, p.dev_status);
+                    PF_EV(2, 7 + 32 * x);
                     if (!ok) return;
                     ++p_count[x];
                     tc_fence_after();
@@ -504,6 +545,7 @@ block_prefill_tc_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_c
                     // released by the epilogue
                     if ((x == 1 || j >= it.nb) && j != steps[x] - 1) mma_commit(bar(B_VEMPTY + st));
                     if (j == steps[x] - 1) mma_commit(bar(B_OFULL + x));
+                    PF_EV(2, 8 + 32 * x);
                 };
                 issue_s(0, 0);
                 if (it.nb > 0) issue_s(1, 0);
@@ -529,6 +571,12 @@ block_prefill_tc_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_c
         uint32_t s_count = 0, o_count = 0;                 // S tiles / O tiles consumed so far by this thread
         uint32_t kv_base = 0;                              // key/value tiles consumed by earlier items
         bool ok = true;
+        PF_EV_DECL;
+#ifdef BT_PF_TRACE
+#define PF_EVS(id) do { if (wq == 0 && lane == 0) PF_EV(x, id); } while (0)
+#else
+#define PF_EVS(id)
+#endif
         for (long long item = blockIdx.x; ok && item < p.n_items; item += gridDim.x) {
             const Item it = decode_item(item, p);
             const int qt = x ? it.qb : it.qa, n_kv = x ? it.nb : it.na;
@@ -540,6 +588,7 @@ block_prefill_tc_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_c
                 const bool diag = (j == qt);
                 ok = mbar_wait(bar(B_SFULL + x), s_count & 1, abort_flag, p.dev_status);  // S_j ready; O settled
                 if (!ok) break;
+                PF_EVS(1);
                 tc_fence_after();
                 // On the diagonal tile the rows of warp w (32w .. 32w+31) see nothing right of column
                 // 32w+31: only column chunks 0..w are loaded and exponentiated, chunk w with a per-row mask.
@@ -552,6 +601,7 @@ block_prefill_tc_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_c
 #pragma unroll
                 for (int c = 0; c < BN / 32; ++c)
                     if (c < nch) tmem_ld_fence32(sr + c * 32);
+                PF_EVS(2);
                 if (diag) {  // masked scores become -inf: they drop out of the maximum and exponentiate to 0
 #pragma unroll
                     for (int c = 0; c < BN / 32; ++c)
@@ -574,6 +624,7 @@ block_prefill_tc_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_c
                     }
                 float mx = fmaxf(fmaxf(mx4[0], mx4[1]), fmaxf(mx4[2], mx4[3]));
                 mx *= p.scale_log2;
+                PF_EVS(3);
                 float factor = 1.f;
                 const bool grow_ref = mx > m_ref + kRescaleThreshold;  // first tile: m_ref = -inf
                 if (grow_ref) {
@@ -638,6 +689,7 @@ block_prefill_tc_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_c
                         tmem_wait_st();
                         tc_fence_before();
                         mbar_arrive(bar(B_P0FULL + x));
+                        PF_EVS(4);
                     }
                 }
                 {
@@ -649,10 +701,12 @@ block_prefill_tc_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_c
                 tmem_wait_st();
                 tc_fence_before();
                 mbar_arrive(bar(B_P1FULL + x));
+                PF_EVS(5);
             }
             if (ok) ok = mbar_wait(bar(B_OFULL + x), o_count & 1, abort_flag, p.dev_status);
             ++o_count;
             if (!ok) break;
+            PF_EVS(6);
             tc_fence_after();
             const float inv = l > 0.f ? 1.f / l : 0.f;
             // O row -> bf16 -> the shared-memory stage that held this tile's last V tile (every MMA that
@@ -679,6 +733,7 @@ block_prefill_tc_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_c
             }
             tc_fence_before();
             asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+            PF_EVS(7);
             asm volatile("barrier.sync.aligned %0, 128;" ::"r"(1 + x) : "memory");  // the warpgroup's 128 rows are staged
             if (wq == 0 && lane == 0) {
                 for (int bx = 0; bx < NB; ++bx)
@@ -687,6 +742,7 @@ block_prefill_tc_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_c
                 asm volatile("cp.async.bulk.wait_group.read 0;" ::: "memory");
                 mbar_arrive(bar(B_VEMPTY + stage_o));
             }
+            PF_EVS(8);
             // the next item's first P V overwrites O: it is issued only after this thread's next
             // arrival on P0FULL, which follows these loads in program order
         }
@@ -775,6 +831,9 @@ static cudaError_t launch_t(const PrefillArgs& a, uint32_t* dev_status, cudaStre
     p.n_classes = (p.n_qtiles + 1) / 2;
     p.n_items = slabs * p.n_classes;
     p.scale_log2 = a.scale_log2;
+#ifdef BT_PF_TRACE
+    p.trace = g_trace;
+#endif
     // one persistent CTA per SM; a grid size coprime to the number of classes makes every CTA
     // cycle through all classes (heavy and light items alike)
     long long grid = p.n_items < sm_count[dev] ? p.n_items : sm_count[dev];
