@@ -24,7 +24,7 @@ import numpy as np
 ROOT = os.path.dirname(os.path.abspath(__file__))
 sys.path.insert(0, ROOT)
 
-from workloads import configs, gen, traffic  # noqa: E402
+from workloads import configs, gen, replicas, traffic  # noqa: E402
 
 METRIC = "decode tokens/s (attention path)"
 FALLBACK_PEAKS = {"hbm_gbs": 6650.0, "bf16_tflops": 1590.0, "bf16_tflops_sustained": 1400.0}
@@ -106,8 +106,7 @@ class ClockSampler:
         return out
 
 
-def dist_env():
-    return int(os.environ.get("RANK", 0)), int(os.environ.get("LOCAL_RANK", 0)), int(os.environ.get("WORLD_SIZE", 1))
+dist_env = replicas.dist_env
 
 
 # ------------------------------------------------------------------------------------------ CPU oracle legs
@@ -229,7 +228,7 @@ def run_gpu(args):
         reduced["n_layers"] = args.layers
     if reduced:  # a smaller copy of the workload, for profiler captures only
         w = configs.scaled(w, **reduced)
-    fill = lambda tid, shape: gen.normal_bf16_device(w.seed + 17 * rank, tid, shape, device="cuda")
+    fill = lambda tid, shape: gen.normal_bf16_device(replicas.replica_seed(w.seed, rank), tid, shape, device="cuda")
     pk = peaks()
 
     def barrier():
@@ -250,12 +249,7 @@ def run_gpu(args):
             step_fn()
         e1.record()
         barrier()
-        ms = e0.elapsed_time(e1) / steps
-        if world > 1:
-            t = torch.tensor([ms], device="cuda")
-            dist.all_reduce(t, op=dist.ReduceOp.MAX)
-            ms = t.item()
-        return ms
+        return replicas.max_over_ranks(e0.elapsed_time(e1) / steps, world, device="cuda")
 
     sampler = ClockSampler(local_rank)
     kern_events = []
@@ -346,7 +340,7 @@ def run_gpu(args):
 
     if rank != 0:
         return 0
-    value = world * tokens_per_step / (ms * 1e-3)
+    value = replicas.job_throughput(tokens_per_step, ms, world)
     if args.workload == "token_decode":
         ms, tokens_per_step = ms * n_tok, tokens_per_step * n_tok  # report the timed unit: one graph replay
     line = {"metric": METRIC, "value": value, "unit": "tokens/s", "n_gpus": world, "steps": args.steps,
@@ -355,7 +349,7 @@ def run_gpu(args):
             "config": workload_config(w, args.workload), "clocks": clocks, "gpu_launches": launches,
             "roofline": roof}
     if ms_e2e is not None:
-        line["e2e"] = {"value": world * tokens_per_step / (ms_e2e * 1e-3), "unit": "tokens/s", "ms_per_step": ms_e2e,
+        line["e2e"] = {"value": replicas.job_throughput(tokens_per_step, ms_e2e, world), "unit": "tokens/s", "ms_per_step": ms_e2e,
                        "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h,
                        "api": "bt_block_decode_step_host (pinned host q,k,v in; out back to host; cache resident)"}
     if world == 1 and args.workload == "block_decode" and not args.no_cpu_baseline and not reduced:
