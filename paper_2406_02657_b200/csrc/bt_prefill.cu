@@ -517,7 +517,7 @@ block_prefill_tc_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_c
                     const uint32_t kc = kv_base + j, st = kc % kKvStages;
                     ok = ok && mbar_wait(bar(B_P0FULL + x), p_count[x] & 1, abort_flag, p.dev_status);
                     PF_EV(2, 4 + 32 * x);
-                    ok = ok && mbar_wait(bar(B_VFULL + st), (kc / kKvStages) & 1, abort_flag, p.dev_status);
+                    // V_j has landed: a softmax thread waited for it before the last arrival on P0FULL
                     PF_EV(2, 5 + 32 * x);
                     if (!ok) return;
                     tc_fence_after();
@@ -581,6 +581,7 @@ block_prefill_tc_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_c
             const Item it = decode_item(item, p);
             const int qt = x ? it.qb : it.qa, n_kv = x ? it.nb : it.na;
             const uint32_t stage_o = (kv_base + n_kv - 1) % kKvStages;  // stage of this tile's last V tile
+            const uint32_t kv0 = kv_base;                  // index of the item's first K/V tile in the rings
             kv_base += it.na;
             if (n_kv == 0) continue;                       // single-tile item: warpgroup B has nothing to do
             float m_ref = kNegInf, l = 0.f;
@@ -688,6 +689,12 @@ block_prefill_tc_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_c
                     if (c == kEarlyChunks - 1) {  // columns 0..95 of P are in place: let their share of P V start
                         tmem_wait_st();
                         tc_fence_before();
+                        // one thread also vouches for V_j: P0FULL then implies "V_j has landed", and the MMA
+                        // thread, whose every barrier round trip leaves the tensor pipe dry, need not ask
+                        if (wq == 0 && lane == 0) {
+                            const uint32_t kc = kv0 + j;
+                            ok = mbar_wait(bar(B_VFULL + kc % kKvStages), (kc / kKvStages) & 1, abort_flag, p.dev_status);
+                        }
                         mbar_arrive(bar(B_P0FULL + x));
                         PF_EVS(4);
                     }
