@@ -75,6 +75,50 @@ __device__ __forceinline__ void fma8(float (&acc)[8], float p, const uint4& r)
     acc[6] = fmaf(p, bf_lo(r.w), acc[6]); acc[7] = fmaf(p, bf_hi(r.w), acc[7]);
 }
 
+// Packed fp32 pairs: one issue slot for two multiply-adds (sm_100).
+__device__ __forceinline__ uint64_t pack2(float lo, float hi)
+{
+    uint64_t d;
+    asm("mov.b64 %0, {%1, %2};" : "=l"(d) : "f"(lo), "f"(hi));
+    return d;
+}
+__device__ __forceinline__ void unpack2(uint64_t v, float& lo, float& hi)
+{
+    asm("mov.b64 {%0, %1}, %2;" : "=f"(lo), "=f"(hi) : "l"(v));
+}
+__device__ __forceinline__ uint64_t ffma2(uint64_t a, uint64_t b, uint64_t c)
+{
+    uint64_t d;
+    asm("fma.rn.f32x2 %0, %1, %2, %3;" : "=l"(d) : "l"(a), "l"(b), "l"(c));
+    return d;
+}
+__device__ __forceinline__ uint64_t fmul2(uint64_t a, uint64_t b)
+{
+    uint64_t d;
+    asm("mul.rn.f32x2 %0, %1, %2;" : "=l"(d) : "l"(a), "l"(b));
+    return d;
+}
+__device__ __forceinline__ uint64_t bf2_to_f2(uint32_t w) { return pack2(bf_lo(w), bf_hi(w)); }
+// q (4 pairs) . row piece (8 bf16); the two halves of the pairs are added at the end
+__device__ __forceinline__ float dot8_x2(const uint64_t (&q2)[4], const uint4& r)
+{
+    uint64_t a = fmul2(q2[0], bf2_to_f2(r.x));
+    a = ffma2(q2[1], bf2_to_f2(r.y), a);
+    a = ffma2(q2[2], bf2_to_f2(r.z), a);
+    a = ffma2(q2[3], bf2_to_f2(r.w), a);
+    float lo, hi;
+    unpack2(a, lo, hi);
+    return lo + hi;
+}
+__device__ __forceinline__ void fma8_x2(uint64_t (&acc2)[4], float p, const uint4& r)
+{
+    const uint64_t p2 = pack2(p, p);
+    acc2[0] = ffma2(p2, bf2_to_f2(r.x), acc2[0]);
+    acc2[1] = ffma2(p2, bf2_to_f2(r.y), acc2[1]);
+    acc2[2] = ffma2(p2, bf2_to_f2(r.z), acc2[2]);
+    acc2[3] = ffma2(p2, bf2_to_f2(r.w), acc2[3]);
+}
+
 // Sum over the LPR consecutive lanes that hold one row (all of them get the total).
 template <int LPR>
 __device__ __forceinline__ float row_sum(float x)

@@ -21,6 +21,9 @@ __device__ __forceinline__ void add_row(SoftmaxState& st, float s, const uint4& 
     st.m = mn;
 }
 
+#ifndef BT_TOK_X2
+#define BT_TOK_X2 1
+#endif
 #ifndef BT_TOK_MINBLOCKS
 #define BT_TOK_MINBLOCKS 3
 #endif
@@ -249,6 +252,12 @@ token_step_pipelined_kernel(TokenArgs a, int seqs_per_cta, int threads_per_seq)
         unpack8(qr, qf);
 #pragma unroll
         for (int d = 0; d < 8; ++d) qf[d] *= a.scale_log2;
+#if BT_TOK_X2
+        const uint64_t q2[4] = {pack2(qf[0], qf[1]), pack2(qf[2], qf[3]), pack2(qf[4], qf[5]), pack2(qf[6], qf[7])};
+#define TOK_DOT(r) dot8_x2(q2, r)
+#else
+#define TOK_DOT(r) dot8(qf, r)
+#endif
         // all scores first (independent dot products and shuffles), then one max, the exponentials
         // and the weighted sum: with at most kMaxRows + 1 rows nothing needs a running rescale
         uint4 vc[kMaxRows];
@@ -258,18 +267,33 @@ token_step_pipelined_kernel(TokenArgs a, int seqs_per_cta, int threads_per_seq)
             const bool v = r < n_old;
             const uint4 kc = v ? my[(size_t)(3 + 2 * r) * kTokThreads] : make_uint4(0, 0, 0, 0);
             vc[r] = v ? my[(size_t)(4 + 2 * r) * kTokThreads] : make_uint4(0, 0, 0, 0);
-            const float d = row_sum<LPR>(dot8(qf, kc));
+            const float d = row_sum<LPR>(TOK_DOT(kc));
             sc[r] = v ? d : kNegInf;
         }
         {
-            const float d = row_sum<LPR>(dot8(qf, kr));
+            const float d = row_sum<LPR>(TOK_DOT(kr));
             sc[kMaxRows] = (b >= 0 && !overflow) ? d : kNegInf;
         }
+#undef TOK_DOT
         float mx = sc[kMaxRows];
 #pragma unroll
         for (int r = 0; r < kMaxRows; ++r) mx = fmaxf(mx, sc[r]);
         float l = 0.f, acc[8] = {0.f, 0.f, 0.f, 0.f, 0.f, 0.f, 0.f, 0.f};
         if (mx != kNegInf) {
+#if BT_TOK_X2
+            uint64_t acc2[4] = {pack2(0.f, 0.f), pack2(0.f, 0.f), pack2(0.f, 0.f), pack2(0.f, 0.f)};
+#pragma unroll
+            for (int r = 0; r < kMaxRows; ++r) {
+                const float pr = ex2(sc[r] - mx);  // 0 for masked rows
+                l += pr;
+                fma8_x2(acc2, pr, vc[r]);
+            }
+            const float pn = ex2(sc[kMaxRows] - mx);
+            l += pn;
+            fma8_x2(acc2, pn, vr);
+#pragma unroll
+            for (int i = 0; i < 4; ++i) unpack2(acc2[i], acc[2 * i], acc[2 * i + 1]);
+#else
 #pragma unroll
             for (int r = 0; r < kMaxRows; ++r) {
                 const float pr = ex2(sc[r] - mx);  // 0 for masked rows
@@ -279,6 +303,7 @@ token_step_pipelined_kernel(TokenArgs a, int seqs_per_cta, int threads_per_seq)
             const float pn = ex2(sc[kMaxRows] - mx);
             l += pn;
             fma8(acc, pn, vr);
+#endif
         }
         if (b >= 0) {
             const size_t slab = (size_t)b * a.H + h;
