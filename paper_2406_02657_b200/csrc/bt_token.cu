@@ -161,6 +161,7 @@ __device__ __forceinline__ void cp_async16(uint32_t dst, const void* src)
 {
     asm volatile("cp.async.cg.shared.global [%0], [%1], 16;" ::"r"(dst), "l"(src) : "memory");
 }
+__device__ __forceinline__ void prefetch_l2(const void* p) { asm volatile("prefetch.global.L2 [%0];" ::"l"(p)); }
 __device__ __forceinline__ void cp_async_commit() { asm volatile("cp.async.commit_group;" ::: "memory"); }
 template <int N>
 __device__ __forceinline__ void cp_async_wait() { asm volatile("cp.async.wait_group %0;" ::"n"(N) : "memory"); }
@@ -198,7 +199,8 @@ token_step_pipelined_kernel(TokenArgs a, int seqs_per_cta, int threads_per_seq)
     };
     // rows of the cache this thread must fetch for a sequence whose length (before the step) is len
     auto rows_to_read = [&](int len) -> int { return (len < 0 || len + 1 > a.cap) ? 0 : len; };
-    auto issue = [&](int i, int len) {
+    // the new row and the query do not depend on the length ...
+    auto issue_new = [&](int i) {
         const int b = seq_of(i);
         if (b >= 0) {
             const int stage = i % kStages;
@@ -206,6 +208,14 @@ token_step_pipelined_kernel(TokenArgs a, int seqs_per_cta, int threads_per_seq)
             cp_async16(slot_addr(stage, 0), reinterpret_cast<const bf16*>(a.q) + slab * HD + sub * 8);
             cp_async16(slot_addr(stage, 1), reinterpret_cast<const bf16*>(a.k_new) + slab * HD + sub * 8);
             cp_async16(slot_addr(stage, 2), reinterpret_cast<const bf16*>(a.v_new) + slab * HD + sub * 8);
+        }
+    };
+    // ... the cached rows to fetch do
+    auto issue_rows = [&](int i, int len) {
+        const int b = seq_of(i);
+        if (b >= 0) {
+            const int stage = i % kStages;
+            const size_t slab = (size_t)b * a.H + h;
             const bf16* cache = reinterpret_cast<const bf16*>(a.kv) + slab * a.cap * 2 * HD + sub * 8;
             const int n = rows_to_read(len);
             for (int r = 0; r < n; ++r) {
@@ -221,18 +231,39 @@ token_step_pipelined_kernel(TokenArgs a, int seqs_per_cta, int threads_per_seq)
     constexpr int kLenAhead = 3, kLens = kDepth + kLenAhead;
     int lens[kLens];
     pdl_launch_dependents();
-    pdl_wait();  // nothing above touched global memory
+    // While the kernel before this one drains, warm L2 with what the first groups will ask for.  A
+    // prefetch returns nothing to the thread, so it is safe ahead of the wait: whatever the previous
+    // kernel still writes reaches L2 as well, and the loads proper come after the wait.
+#pragma unroll
+    for (int d = 0; d < kDepth + 1; ++d) {
+        const int b = seq_of(d);
+        if (b >= 0) {
+            const size_t slab = (size_t)b * a.H + h;
+            if ((sub & 7) == 0) {  // one request per 128-byte line
+                prefetch_l2(reinterpret_cast<const bf16*>(a.q) + slab * HD + sub * 8);
+                prefetch_l2(reinterpret_cast<const bf16*>(a.k_new) + slab * HD + sub * 8);
+                prefetch_l2(reinterpret_cast<const bf16*>(a.v_new) + slab * HD + sub * 8);
+            }
+            if (within == 0) prefetch_l2(a.len + b);
+        }
+    }
+    pdl_wait();  // nothing above read or wrote global memory
+    // prologue: the first groups' q, k_new, v_new are requested before their lengths are known, so the
+    // two DRAM round trips (length, then rows) overlap with them
+#pragma unroll
+    for (int d = 0; d < kDepth; ++d) issue_new(d);
 #pragma unroll
     for (int d = 0; d < kLens; ++d) lens[d] = load_len(seq_of(d));
 #pragma unroll
     for (int d = 0; d < kDepth; ++d) {
-        issue(d, lens[d]);
-        cp_async_commit();
+        issue_rows(d, lens[d]);
+        cp_async_commit();   // group d: its rows (and, in the first group, every q, k_new, v_new above)
     }
 
     for (int i = 0; i < n_iter; ++i) {
         const int len_ahead = load_len(seq_of(i + kLens));
-        issue(i + kDepth, lens[kDepth]);
+        issue_new(i + kDepth);
+        issue_rows(i + kDepth, lens[kDepth]);
         cp_async_commit();
         cp_async_wait<kDepth>();  // the copies of group i have landed
 
