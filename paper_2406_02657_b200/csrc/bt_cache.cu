@@ -19,6 +19,14 @@ __global__ void __launch_bounds__(kAppendThreads) kv_append_kernel(CacheView c, 
     const int b = blockIdx.x;
     if (kFused) {  // launched with launch_pdl
         pdl_launch_dependents();
+        // warm L2 with the length and the rows to copy while the kernel before this one drains
+        // (a prefetch returns nothing to the thread, so it is safe ahead of the wait)
+        if (threadIdx.x == 0) asm volatile("prefetch.global.L2 [%0];" ::"l"(c.len + b));
+        const size_t bytes = (size_t)H * n_new * hd * 2;
+        for (size_t o = (size_t)threadIdx.x * 128; o < bytes; o += (size_t)blockDim.x * 128) {
+            asm volatile("prefetch.global.L2 [%0];" ::"l"(reinterpret_cast<const char*>(k_new) + (size_t)b * bytes + o));
+            asm volatile("prefetch.global.L2 [%0];" ::"l"(reinterpret_cast<const char*>(v_new) + (size_t)b * bytes + o));
+        }
         pdl_wait();
     }
     const int len = c.len[b];

@@ -134,13 +134,28 @@ __global__ void __launch_bounds__(kThreads, 1) block_decode_ring_kernel(DecodeAr
     uint64_t policy;
     asm volatile("createpolicy.fractional.L2::evict_first.b64 %0, 1.0;" : "=l"(policy));
     pdl_launch_dependents();
-    pdl_wait();  // nothing above touched global memory
 
     const int n_items = a.B * a.H * a.splits;
     const int stride = kWarps * gridDim.x;
     const int first = warp * gridDim.x + blockIdx.x;   // neighbouring items go to different SMs
     const bf16* Kall = reinterpret_cast<const bf16*>(a.k);
     const bf16* Vall = reinterpret_cast<const bf16*>(a.v);
+    // While the kernel before this one drains, warm L2 with the first ring-full of this warp's first
+    // item (rows 0.. of its slab, whatever its length turns out to be: the rows exist either way), its
+    // length and its query.  A prefetch returns nothing to the thread, so it is safe ahead of the wait.
+    if (first < n_items && a.splits == 1) {
+        const size_t off = (size_t)first * a.n_max * HD;
+        const int lines = min(kStages * G::CHUNK_BYTES, a.n_max * G::ROW_BYTES) / 128;  // 128-byte lines to touch
+        for (int i = lane; i < lines; i += 32) {
+            asm volatile("prefetch.global.L2 [%0];" ::"l"(reinterpret_cast<const char*>(Kall + off) + (size_t)i * 128));
+            asm volatile("prefetch.global.L2 [%0];" ::"l"(reinterpret_cast<const char*>(Vall + off) + (size_t)i * 128));
+        }
+        if (lane == 0) {
+            asm volatile("prefetch.global.L2 [%0];" ::"l"(a.len + first / a.H));
+            asm volatile("prefetch.global.L2 [%0];" ::"l"(reinterpret_cast<const bf16*>(a.q) + (size_t)first * HD));
+        }
+    }
+    pdl_wait();  // nothing above read or wrote global memory
 
     // ---- producer cursor (kept by every lane, acted on by lane 0): next chunk to request
     int p_item = first, p_c = 0, p_nchunks = 0;
