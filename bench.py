@@ -316,10 +316,13 @@ def run_gpu(args):
     else:
         run = harness.PrefillRun(w, fill=fill)
         tokens_per_step = w.batch * w.prompt_tokens
+        # a bench step = one CUDA-graph replay of the 12 launches (all of the same kernel, overlapping their
+        # neighbours' ramp and drain through programmatic dependent launch); per-launch time = step time / 12
+        run.capture()
         sampler.start()
-        ms = timed(lambda: run.step(kern_events), lambda: None, args.steps, args.warmup)
+        ms = timed(run.replay, lambda: None, args.steps, args.warmup)
         clocks = sampler.stop()
-        kern_events = kern_events[args.warmup * w.n_layers:]
+        kern_events = []
         ms_e2e, h2d, d2h = None, 0, 0
         alg_bytes = traffic.prefill_layer_bytes(w.batch, w.heads, w.prompt_blocks, w.head_dim)
         dom = "block_prefill_kernel"

@@ -115,6 +115,12 @@ __device__ __forceinline__ void tma_load_3d(uint32_t dst, const CUtensorMap* map
         : "memory");
 }
 
+// Ask for a tile to be brought into L2 (no shared-memory destination, nothing to wait for).
+__device__ __forceinline__ void tma_prefetch_l2_3d(const CUtensorMap* map, int c0, int c1, int c2)
+{
+    asm volatile("cp.async.bulk.prefetch.tensor.3d.L2.global.tile [%0, {%1, %2, %3}];" ::"l"(map), "r"(c0), "r"(c1), "r"(c2) : "memory");
+}
+
 // Tile store shared -> global (rows outside the tensor are dropped), as one bulk group of this thread.
 __device__ __forceinline__ void tma_store_3d(const CUtensorMap* map, uint32_t src, int c0, int c1, int c2)
 {
@@ -426,6 +432,26 @@ block_prefill_tc_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_c
     __syncthreads();
     tc_fence_after();
     const uint32_t tmem = *tmem_slot;
+
+    // Programmatic dependent launch: this CTA may have been placed while the kernel before it in the
+    // stream drains.  Until that kernel is done only L2 prefetches are issued (they return nothing to
+    // the thread): the first item's Q tiles and its first K and V tiles.
+    pdl_launch_dependents();
+    if (warp == kProducerWarp && lane == 0 && (long long)blockIdx.x < p.n_items) {
+        asm volatile("prefetch.tensormap [%0];" ::"l"(&mapQ) : "memory");
+        asm volatile("prefetch.tensormap [%0];" ::"l"(&mapK) : "memory");
+        asm volatile("prefetch.tensormap [%0];" ::"l"(&mapV) : "memory");
+        const Item it = decode_item(blockIdx.x, p);
+        for (int bx = 0; bx < NB; ++bx) {
+            tma_prefetch_l2_3d(&mapQ, bx * 64, it.qa * BM, it.bh);
+            if (it.nb > 0) tma_prefetch_l2_3d(&mapQ, bx * 64, it.qb * BM, it.bh);
+            for (int j = 0; j < it.na && j < kKvStages; ++j) {
+                tma_prefetch_l2_3d(&mapK, bx * 64, j * BN, it.bh);
+                tma_prefetch_l2_3d(&mapV, bx * 64, j * BN, it.bh);
+            }
+        }
+    }
+    pdl_wait();
 
     if (warp == kProducerWarp) {
         // ------------------------------------------------------------------ TMA producer
@@ -845,8 +871,7 @@ static cudaError_t launch_t(const PrefillArgs& a, uint32_t* dev_status, cudaStre
     // cycle through all classes (heavy and light items alike)
     long long grid = p.n_items < sm_count[dev] ? p.n_items : sm_count[dev];
     while (grid > 1 && p.n_items > grid && gcd_int((int)grid, p.n_classes) != 1) --grid;
-    block_prefill_tc_kernel<HD><<<(unsigned)grid, kThreads, smem_bytes<HD>(), stream>>>(mq, mk, mv, mo, p);
-    return cudaGetLastError();
+    return launch_pdl(block_prefill_tc_kernel<HD>, dim3((unsigned)grid), dim3(kThreads), (size_t)smem_bytes<HD>(), stream, mq, mk, mv, mo, p);
 }
 
 }  // namespace pf

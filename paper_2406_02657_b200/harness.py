@@ -174,10 +174,29 @@ class PrefillRun:
         self.out = torch.empty(shape, dtype=torch.bfloat16, device=device)
         self.launches_per_step = w.n_layers
 
-    def step(self, events=None):
+    def capture(self):
+        """One step as two CUDA graphs: a plain one (replay) and a twin with (external) timing events
+        around every launch (replay_timed; afterwards graph_events hold that replay's times)."""
+        self.step()
+        torch.cuda.synchronize()
+        self.graph = torch.cuda.CUDAGraph()
+        with torch.cuda.graph(self.graph):
+            self.step()
+        self.graph_events = []
+        self.graph_timed = torch.cuda.CUDAGraph()
+        with torch.cuda.graph(self.graph_timed):
+            self.step(self.graph_events, external=True)
+
+    def replay(self):
+        self.graph.replay()
+
+    def replay_timed(self):
+        self.graph_timed.replay()
+
+    def step(self, events=None, external=False):
         for l in range(self.w.n_layers):
             if events is not None:
-                e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+                e0, e1 = torch.cuda.Event(enable_timing=True, external=external), torch.cuda.Event(enable_timing=True, external=external)
                 e0.record()
             bt.bt_block_prefill_attn(self.cfg, self.q[l], self.k[l], self.v[l], self.out[l], n_blocks=self.w.prompt_blocks)
             if events is not None:
