@@ -72,15 +72,24 @@ class BlockDecodeStep:
         return g
 
     def capture(self):
-        """Capture rewind + one whole step into two CUDA graphs: a plain one (replay) and one with
-        timing events (external, so that they may sit inside a graph) around every attention launch
-        (replay_timed; after it the events hold that replay's per-launch times)."""
+        """Capture rewind + one whole step into CUDA graphs: a plain one (replay), one with timing events
+        (external, so that they may sit inside a graph) around every attention launch (replay_timed;
+        after it the events hold that replay's per-launch times), and the attention launches alone
+        (replay_attn)."""
         self.step()  # anything lazy (module load, per-device set-up) happens outside the capture
         self.rewind()
         torch.cuda.synchronize()
         self.graph = self._capture(None)
         self.graph_events = []
         self.graph_timed = self._capture(self.graph_events)
+        # the attention launches alone (lengths as a step leaves them: ctx_blocks rows), for their own time
+        self.graph_attn = torch.cuda.CUDAGraph()
+        with torch.cuda.graph(self.graph_attn):
+            for l in range(self.w.n_layers):
+                bt.bt_block_decode_attn(self.cfg, self.cache, l, self.q[l], self.out[l], self.ws, dev_status=self.status)
+
+    def replay_attn(self):
+        self.graph_attn.replay()
 
     def replay_timed(self):
         self.graph_timed.replay()
