@@ -1,8 +1,7 @@
-// Block-decoder decode attention (paper section 2.3; appendix E.2): one query per
-// (sequence, head) over the cached block rows, memory-bound.  Each CTA streams a contiguous
-// range of K and V rows with 128-bit read-once loads, keeps an online softmax per lane and
-// merges lanes, warps and (when the row range is split across CTAs) splits with the
-// log-sum-exp rule.
+// Block-decoder decode attention, second half (paper section 2.3; appendix E.2): the streaming kernel
+// lives in bt_decode_ring.cu; here are the merge of the per-split partial results by the log-sum-exp
+// rule, and the plain CUDA-core prefill kernel (one query block per CTA over rows 0..t, 128-bit
+// read-once loads, online softmax per lane) that serves shapes the tensor-core kernel does not take.
 #include "bt_common.cuh"
 #include "bt_kernels.h"
 

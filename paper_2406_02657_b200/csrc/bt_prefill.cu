@@ -1,21 +1,25 @@
 // Block-decoder prefill attention on the 5th-generation tensor cores (paper sections 2.1, 2.3:
 // the prefill stage processes all prompt blocks in parallel; causal over blocks).
 //
-// One CTA owns 128 query blocks of one (sequence, head) and walks the key/value blocks
-// 0 .. diagonal in tiles of 128; two CTAs share an SM (96 KB of shared memory and 256 tensor-
-// memory columns each), so one CTA's softmax overlaps the other's MMAs and loads:
-//   warp 4 (one lane): TMA producer and tcgen05.mma issuer - Q once, then per tile S = Q K^T into
-//                      tensor memory and O += P V with P read from tensor memory (the probabilities
-//                      never visit shared memory); K_j+1 is requested as soon as S_j has consumed
-//                      K_j, V_j+1 as soon as P_j V_j has consumed V_j
-//   warps 0-3        : softmax - each thread owns one query row (= one TMEM lane) and holds its
-//                      128 scores in registers: one batch of tensor-memory loads, row maximum,
-//                      exp2 (packed fp32x2 multiply-adds around it), bf16 P written over the S
-//                      columns, running row sum; on the diagonal tile a warp skips the column
-//                      chunks that are masked for all of its rows.  O is rescaled in TMEM only when
-//                      the row maximum grew by more than 2^8 (otherwise the old reference is kept,
-//                      exact because O and the row sum share it)
-// All waits are bounded: a wait that runs out raises BT_DEV_TIMEOUT and the CTA winds down.
+// Persistent kernel, one CTA per SM (all of its shared memory and its 512 tensor-memory columns).
+// A work item is a pair of neighbouring 128-row query tiles of one (sequence, head); the two tiles
+// walk the same key/value tiles 0 .. diagonal, so K and V are loaded once for both.  Roles:
+//   warps 0-3 / 4-7 : softmax of query tile A / B - each thread owns one query row (= one TMEM lane)
+//                     and holds its 128 scores in registers: one batch of tensor-memory loads, row
+//                     maximum, exp2 (packed fp32x2 multiply-adds around it), bf16 P written over the S
+//                     columns (signalled in two parts), running row sum; on the diagonal tile a warp
+//                     skips the column chunks that are masked for all of its rows.  O is rescaled in
+//                     TMEM only when the row maximum grew by more than 2^8 (otherwise the old
+//                     reference is kept, exact because O and the row sum share it).  At the end of an
+//                     item the rows go through shared memory (the stage of the tile's last V tile)
+//                     to a TMA store.
+//   warp 8 (1 lane) : TMA producer - Q tiles (Q_A double-buffered an item ahead), K and V rings of
+//                     two stages, 128-byte swizzle
+//   warp 9 (1 lane) : tcgen05.mma issuer - S = Q K^T into tensor memory, O += P V with P read from
+//                     tensor memory (the probabilities never visit shared memory), in the order
+//                     PV_A(j) S_A(j+1) PV_B(j) S_B(j+1): the tensor pipe works for one tile while the
+//                     other tile is in its softmax
+// All waits are bounded in wall time: one that runs out raises BT_DEV_TIMEOUT and the CTA winds down.
 #include <cuda.h>
 
 #include "bt_common.cuh"
@@ -290,33 +294,6 @@ __device__ __forceinline__ float fmax3(float a, float b, float c)
     return d;
 }
 
-__device__ __forceinline__ uint64_t fadd2_rm(uint64_t a, uint64_t b)
-{
-    uint64_t d;
-    asm("add.rm.f32x2 %0, %1, %2;" : "=l"(d) : "l"(a), "l"(b));
-    return d;
-}
-// 2^x for two values on the FMA and integer pipes (no special-function unit): x = n + f with
-// n = floor(x), f in [0,1); 2^f by a cubic with maximum relative error 8.6e-5 (well below the bf16
-// rounding the result gets), then n is added to the exponent field.  x is clamped at -127 (result
-// 2^-127 flushes to 0 in the bf16 product); x must stay below 128.
-__device__ __forceinline__ void exp2_poly2(float x0, float x1, float& p0, float& p1)
-{
-    const float kMagic = 12582912.f;  // 1.5 * 2^23: adding it with round-down leaves floor(x) in the low mantissa bits
-    const uint64_t x = pack2(fmaxf(x0, -127.f), fmaxf(x1, -127.f));
-    const uint64_t t = fadd2_rm(x, pack2(kMagic, kMagic));
-    const uint64_t fl = fadd2(t, pack2(-kMagic, -kMagic));
-    const uint64_t f = ffma2(fl, pack2(-1.f, -1.f), x);
-    uint64_t q = ffma2(f, pack2(0.07706617563962936f, 0.07706617563962936f), pack2(0.22764593362808228f, 0.22764593362808228f));
-    q = ffma2(q, f, pack2(0.6951165795326233f, 0.6951165795326233f));
-    q = ffma2(q, f, pack2(1.f, 1.f));
-    float t0, t1, q0, q1;
-    unpack2(t, t0, t1);
-    unpack2(q, q0, q1);
-    p0 = __uint_as_float(__float_as_uint(q0) + (__float_as_uint(t0) << 23));
-    p1 = __uint_as_float(__float_as_uint(q1) + (__float_as_uint(t1) << 23));
-}
-
 // Work decomposition.  The T query blocks of one (sequence, head) form n = ceil(T/128) query tiles;
 // tile t needs key/value tiles 0..t.  An item is a pair of neighbouring query tiles taken from the
 // top: class k holds tiles A = n-1-2k (na = n-2k tile steps) and B = n-2-2k (nb = na-1 steps; absent
@@ -343,13 +320,9 @@ long long* g_trace = nullptr;
 constexpr int kProducerWarp = 8, kMmaWarp = 9;
 constexpr int kThreads = 320;
 constexpr int kKvStages = 2;
-#ifndef BT_PF_POLY_OF8
-#define BT_PF_POLY_OF8 0
-#endif
 #ifndef BT_PF_EARLY_CHUNKS
 #define BT_PF_EARLY_CHUNKS 3
 #endif
-constexpr int kPolyOf8 = BT_PF_POLY_OF8;                 // exponentials per 8 computed without the special-function unit (0,2,4,6,8)
 constexpr int kEarlyChunks = BT_PF_EARLY_CHUNKS;             // 32-column chunks of P signalled ahead of the rest
 constexpr int kQBufs = 3;                   // Q_A alternates between buffers 0 and 2, Q_B lives in buffer 1
 
@@ -690,12 +663,8 @@ block_prefill_tc_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_c
                         }
 #pragma unroll
                         for (int i = 0; i < 32; i += 2) {
-                            // kPolyOf8 of every 8 exponentials go to the FMA pipes, the rest to the special-function unit
-                            float p0, p1;
-                            if (((i >> 1) & 3) < kPolyOf8 / 2) exp2_poly2(__uint_as_float(sr[c * 32 + i]), __uint_as_float(sr[c * 32 + i + 1]), p0, p1);
-                            else { p0 = ex2(__uint_as_float(sr[c * 32 + i])); p1 = ex2(__uint_as_float(sr[c * 32 + i + 1])); }
-                            sr[c * 32 + i] = __float_as_uint(p0);
-                            sr[c * 32 + i + 1] = __float_as_uint(p1);
+                            sr[c * 32 + i] = __float_as_uint(ex2(__uint_as_float(sr[c * 32 + i])));
+                            sr[c * 32 + i + 1] = __float_as_uint(ex2(__uint_as_float(sr[c * 32 + i + 1])));
                         }
 #pragma unroll
                         for (int i = 0; i < 32; i += 4) {
