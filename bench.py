@@ -230,6 +230,8 @@ def run_gpu(args):
         reduced["batch"] = args.batch
     if args.layers:
         reduced["n_layers"] = args.layers
+    if args.prefix_len and args.workload == "token_decode" and args.prefix_len != w.prefix_len:
+        w = configs.scaled(w, prefix_len=args.prefix_len)
     if reduced:  # a smaller copy of the workload, for profiler captures only
         w = configs.scaled(w, **reduced)
     fill = lambda tid, shape: gen.normal_bf16_device(replicas.replica_seed(w.seed, rank), tid, shape, device="cuda")
@@ -296,7 +298,9 @@ def run_gpu(args):
         assert run.status.item() == 0
         ms = ms_graph / n_tok
         ms_e2e, h2d, d2h = None, 0, 0
-        alg_bytes = sum(traffic.token_decode_layer_bytes(w.batch, w.heads, w.head_dim, j) for j in range(w.block_len)) / w.block_len
+        P = w.prefix_len  # step 0 appends the P prefix rows, step j >= 1 one row over P + j - 1 cached rows
+        alg_bytes = (traffic.token_decode_layer_bytes(w.batch, w.heads, w.head_dim, 0, P) +
+                     sum(traffic.token_decode_layer_bytes(w.batch, w.heads, w.head_dim, P + j - 1) for j in range(1, w.block_len))) / w.block_len
         dom = "token_step_pipelined_kernel"
         launches = run.launches_per_step * n_tok * args.steps
         step_bytes = w.n_layers * alg_bytes
@@ -392,6 +396,7 @@ def main():
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--workload", default="block_decode", choices=["block_decode", "token_decode", "block_prefill", "block_prefill_8k", "sweep"])
     ap.add_argument("--block-len", type=int, default=4, help="L_B of the generation sweep (1, 2, 4 or 8)")
+    ap.add_argument("--prefix-len", type=int, default=0, help="token_decode: prefix length P (default 1 = BASELINE configs[2]; 2 = the paper's main setting)")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--batch", type=int, default=0, help="override the batch (profiling a small case; not a bench number)")
     ap.add_argument("--layers", type=int, default=0, help="override the layer count (profiling a small case)")

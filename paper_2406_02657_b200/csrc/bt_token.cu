@@ -42,6 +42,8 @@ __global__ void __launch_bounds__(256, BT_TOK_MINBLOCKS) token_decode_kernel(Tok
     const int b = blockIdx.x * seqs_per_cta + sic;
     const bool active = sic < seqs_per_cta && b < a.B;
 
+    pdl_launch_dependents();  // launched with launch_pdl
+    pdl_wait();               // nothing above touched global memory
     const bool appended = a.k_new != nullptr;
     const bool fast = a.n_q == 1 && appended;
     const size_t slab = active ? (size_t)b * a.H + h : 0;
@@ -104,6 +106,58 @@ __global__ void __launch_bounds__(256, BT_TOK_MINBLOCKS) token_decode_kernel(Tok
 #pragma unroll
             for (int i = 0; i < 8; ++i) o[i] = st.acc[i] * inv;
             *reinterpret_cast<uint4*>(op) = pack8(o);
+        }
+    } else if (appended && a.reset_first && a.reset_mask == nullptr && a.n_q <= 4) {
+        // block start (section 2.4): every sequence is reset and the P prefix rows arrive together.  There
+        // is nothing cached to read: all 3 P rows are requested at once and stay in registers, query i
+        // attends to the new rows 0..i.
+        constexpr int kMaxQ = 4;
+        uint4 qn[kMaxQ], kn[kMaxQ], vn[kMaxQ];
+#pragma unroll
+        for (int i = 0; i < kMaxQ; ++i) {
+            const bool v = active && i < a.n_q;
+            qn[i] = v ? ld_stream(qp + (size_t)i * HD) : make_uint4(0, 0, 0, 0);
+            kn[i] = v ? ld_stream(kp + (size_t)i * HD) : make_uint4(0, 0, 0, 0);
+            vn[i] = v ? ld_stream(vp + (size_t)i * HD) : make_uint4(0, 0, 0, 0);
+        }
+        const bool write = active && !overflow;  // overflow here means n_q > capacity: refused on the host already
+#pragma unroll
+        for (int i = 0; i < kMaxQ; ++i) {
+            if (i < a.n_q) {  // uniform
+                float qf[8];
+                unpack8(qn[i], qf);
+#pragma unroll
+                for (int d = 0; d < 8; ++d) qf[d] *= a.scale_log2;
+                float sc[kMaxQ];
+                float mx = kNegInf;
+#pragma unroll
+                for (int j = 0; j < kMaxQ; ++j) {
+                    if (j <= i) {
+                        sc[j] = row_sum<LPR>(dot8(qf, kn[j]));
+                        mx = fmaxf(mx, sc[j]);
+                    }
+                }
+                float l = 0.f, acc[8] = {0.f, 0.f, 0.f, 0.f, 0.f, 0.f, 0.f, 0.f};
+#pragma unroll
+                for (int j = 0; j < kMaxQ; ++j) {
+                    if (j <= i) {
+                        const float pj = ex2(sc[j] - mx);
+                        l += pj;
+                        fma8(acc, pj, vn[j]);
+                    }
+                }
+                if (active) {
+                    float o[8];
+                    const float inv = write ? 1.f / l : 0.f;
+#pragma unroll
+                    for (int d = 0; d < 8; ++d) o[d] = acc[d] * inv;
+                    *reinterpret_cast<uint4*>(op + (size_t)i * HD) = pack8(o);
+                }
+                if (write) {
+                    *reinterpret_cast<uint4*>(cache + (size_t)i * 2 * HD) = kn[i];
+                    *reinterpret_cast<uint4*>(cache + (size_t)i * 2 * HD + HD) = vn[i];
+                }
+            }
         }
     } else {
         // general step: n_q rows (the P prefix rows at a block start), or attend-only.
@@ -411,6 +465,9 @@ cudaError_t launch_token_decode(const TokenArgs& a, cudaStream_t stream)
         if (a.cap - 1 <= 4)
             return a.hd == 64 ? launch_pipelined<64, BT_TOK_DEPTH4, 4, BT_TOK_CTAS4>(a, spc_p, tps, stream)
                               : launch_pipelined<128, BT_TOK_DEPTH4, 4, BT_TOK_CTAS4>(a, spc_p, tps, stream);
+        if (a.cap - 1 <= 5)  // e.g. L_B = 4 with the paper's main prefix length P = 2: still two CTAs per SM
+            return a.hd == 64 ? launch_pipelined<64, 1, 5, 2>(a, spc_p, tps, stream)
+                              : launch_pipelined<128, 1, 5, 2>(a, spc_p, tps, stream);
         return a.hd == 64 ? launch_pipelined<64, 1, 8, 1>(a, spc_p, tps, stream)
                           : launch_pipelined<128, 1, 8, 1>(a, spc_p, tps, stream);
     }
@@ -419,11 +476,8 @@ cudaError_t launch_token_decode(const TokenArgs& a, cudaStream_t stream)
     if (spc > a.B) spc = a.B;
     const int threads = ((spc * tps + 31) / 32) * 32;
     const int grid = (a.B + spc - 1) / spc;
-    if (a.hd == 64)
-        token_decode_kernel<64><<<grid, threads, 0, stream>>>(a, spc, tps);
-    else
-        token_decode_kernel<128><<<grid, threads, 0, stream>>>(a, spc, tps);
-    return cudaGetLastError();
+    return a.hd == 64 ? launch_pdl(token_decode_kernel<64>, dim3(grid), dim3(threads), 0, stream, a, spc, tps)
+                      : launch_pdl(token_decode_kernel<128>, dim3(grid), dim3(threads), 0, stream, a, spc, tps);
 }
 
 }  // namespace bt

@@ -117,35 +117,45 @@ class BlockDecodeStep:
 
 
 class TokenDecodeRun:
-    """Token-decoder steps over all layers (section 2.4): step j of a block resets (j == 0),
-    appends one row and attends over the local cache (prefix + tokens of the same block)."""
+    """Token-decoder steps over all layers (section 2.4): step 0 of a block resets the local cache and
+    appends the P prefix rows (P queries, causal among themselves), step j >= 1 appends the row of the
+    token produced by step j-1; every step attends over the local cache (prefix + tokens of the same
+    block)."""
 
     def __init__(self, w, device="cuda", fill=None, ring=8):
         self.w, self.device = w, device
         self.cfg = bt.make_config(w.batch, w.heads, w.head_dim, w.block_len, w.prefix_len, max(1, w.max_blocks), w.n_layers)
         self.cache = bt.LocalCache(self.cfg, device)
-        io = (ring, w.n_layers, w.batch, w.heads, 1, w.head_dim)
+        P = w.prefix_len
+        io = (ring, w.n_layers, w.batch, w.heads, P, w.head_dim)  # step 0 of a block uses all P rows, later steps row 0
         mk = (lambda tid: fill(tid, io)) if fill is not None else (lambda tid: torch.zeros(io, dtype=torch.bfloat16, device=device))
         self.q, self.k_new, self.v_new = mk(5), mk(6), mk(7)
         self.out = torch.empty(io[1:], dtype=torch.bfloat16, device=device)
+        # contiguous one-row views for the steps after the first (the library takes [B][H][n][hd] contiguous)
+        if P > 1:
+            self.q1, self.k1, self.v1 = (t[:, :, :, :, :1].contiguous() for t in (self.q, self.k_new, self.v_new))
+            self.out1 = torch.empty((w.n_layers, w.batch, w.heads, 1, w.head_dim), dtype=torch.bfloat16, device=device)
+        else:
+            self.q1, self.k1, self.v1, self.out1 = self.q, self.k_new, self.v_new, self.out
         self.status = torch.zeros(1, dtype=torch.int32, device=device)
         self.ring = ring
         self.t = 0
         self.launches_per_step = w.n_layers
 
     def token_step(self, events=None):
-        """Token step t (prefix length 1: the prefix row is the first row of each block).  events: optional
-        list receiving an (external) timing event pair around every launch."""
+        """Token step t.  events: optional list receiving an (external) timing event pair around every launch."""
         w = self.w
         j = self.t % w.block_len
         r = self.t % self.ring
+        first = j == 0
+        q, k, v, out = (self.q, self.k_new, self.v_new, self.out) if first else (self.q1, self.k1, self.v1, self.out1)
         for l in range(w.n_layers):
             if events is not None:
                 e0 = torch.cuda.Event(enable_timing=True, external=True)
                 e1 = torch.cuda.Event(enable_timing=True, external=True)
                 e0.record()
-            bt.bt_token_decode_attn(self.cfg, self.cache, l, self.q[r, l], self.k_new[r, l], self.v_new[r, l], self.out[l],
-                                    n_q=1, reset_first=(j == 0), dev_status=self.status)
+            bt.bt_token_decode_attn(self.cfg, self.cache, l, q[r, l], k[r, l], v[r, l], out[l],
+                                    n_q=(w.prefix_len if first else 1), reset_first=first, dev_status=self.status)
             if events is not None:
                 e1.record()
                 events.append((e0, e1))

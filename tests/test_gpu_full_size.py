@@ -80,6 +80,34 @@ def test_token_decode_full_size_two_blocks(bt):
     assert run.status.item() == 0
 
 
+def test_token_decode_full_batch_prefix_length_two(bt):
+    """The paper's main setting P = 2 at the full batch: a block starts with a two-row causal prefix step."""
+    from paper_2406_02657_b200 import harness
+    w = configs.scaled(configs.TOKEN_DECODE, prefix_len=2, n_layers=2)
+    run = harness.TokenDecodeRun(w, fill=_fill(w))
+    seqs = [0, 7, 2048, 4095]
+    ocache = {l: oracle.Cache(len(seqs), w.heads, w.local_cap, w.head_dim) for l in range(w.n_layers)}
+    n_steps = 2 * w.block_len
+    sched = schedule.token_step_schedule(w.block_len, w.prefix_len, n_steps)
+    for t in range(n_steps):
+        r = t % run.ring
+        first = t % w.block_len == 0
+        run.token_step()
+        torch.cuda.synchronize()
+        reset, n_app, len_after = sched[t]
+        assert n_app == (w.prefix_len if first else 1)
+        assert (run.cache.len == len_after).all(), f"step {t}: lengths differ from the schedule model"
+        src = (run.q, run.k_new, run.v_new, run.out) if first else (run.q1, run.k1, run.v1, run.out1)
+        for l in range(w.n_layers):
+            q, k, v = (gen.torch_to_bits(x[r, l][seqs]) for x in src[:3])
+            ref = oracle.token_decode_attn(ocache[l], q, k, v, reset_first=bool(reset))
+            assert_close(src[3][l][seqs], ref, f"P=2 token step {t} layer {l}")
+            gk, gv = local_kv_split(run.cache.kv[l][seqs])
+            assert np.array_equal(gk[:, :, :len_after], ocache[l].k[:, :, :len_after])
+            assert np.array_equal(gv[:, :, :len_after], ocache[l].v[:, :, :len_after])
+    assert run.status.item() == 0
+
+
 def test_block_prefill_full_size(bt):
     """BASELINE configs[3]: batch 32, 512 prompt blocks, 16 heads, head_dim 128, 12 layers."""
     from paper_2406_02657_b200 import harness
