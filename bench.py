@@ -377,7 +377,7 @@ def run_gpu(args):
     if ms_e2e is not None:
         line["e2e"] = {"value": replicas.job_throughput(tokens_per_step, ms_e2e, world), "unit": "tokens/s", "ms_per_step": ms_e2e,
                        "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h,
-                       "api": "bt_block_decode_step_host (pinned host q,k,v in; out back to host; cache resident)"}
+                       "api": "bt_block_decode_step_host, one call per layer spread over 3 streams (pinned host q,k,v in; out back to host; cache resident)"}
     if world == 1 and args.workload == "block_decode" and not args.no_cpu_baseline and not reduced:
         line["cpu_baseline"] = cpu_baseline_block_decode(w, run)
     if reduced:

@@ -109,11 +109,29 @@ class BlockDecodeStep:
         one = self.w.batch * self.w.heads * self.w.head_dim * 2
         return 3 * one * self.w.n_layers, one * self.w.n_layers
 
-    def step_host(self):
+    def step_host(self, n_streams=3):
+        """The step through bt_block_decode_step_host, one call per layer.  The layers' inputs all come from
+        the host, so the calls are independent: they are spread round-robin over a few streams (forked from
+        and joined back into the current one), which lets one layer's host-device copies run under another
+        layer's kernels.  Each stream has its own workspace (the calls of one stream are ordered)."""
         h = self._host_buffers()
+        main = torch.cuda.current_stream()
+        if getattr(self, "_side", None) is None or len(self._side) != n_streams:
+            self._side = [torch.cuda.Stream() for _ in range(n_streams)]
+            self._side_ws = [bt.alloc_workspace(self.cfg, self.device) for _ in range(n_streams)]
+            self._fork = torch.cuda.Event()
+            self._join = [torch.cuda.Event() for _ in range(n_streams)]
+        self._fork.record(main)
+        for s in self._side:
+            s.wait_event(self._fork)
         for l in range(self.w.n_layers):
+            i = l % n_streams
             bt.bt_block_decode_step_host(self.cfg, self.cache, l, h["q"][l], h["k"][l], h["v"][l], h["out"][l],
-                                         h["qd"][l], h["kd"][l], h["vd"][l], self.out[l], self.ws, dev_status=self.status)
+                                         h["qd"][l], h["kd"][l], h["vd"][l], self.out[l], self._side_ws[i], dev_status=self.status,
+                                         stream=self._side[i])
+        for s, e in zip(self._side, self._join):
+            e.record(s)
+            main.wait_event(e)
 
 
 class TokenDecodeRun:
