@@ -52,6 +52,26 @@ def test_block_decode_step_full_size(bt):
         assert_close(run.out[l][seqs][:, :, 0], ref, f"full-size block decode layer {l}")
 
 
+def test_block_decode_step_through_host_buffers(bt):
+    """The e2e path of bench.py: the same step driven from pinned host buffers through
+    bt_block_decode_step_host (per-layer calls on several streams) gives the device-resident step's
+    outputs bit for bit, and the same cache."""
+    from paper_2406_02657_b200 import harness
+    w = configs.scaled(configs.BLOCK_DECODE, batch=64, n_layers=5)
+    run = harness.BlockDecodeStep(w, fill=_fill(w))
+    run.step()
+    torch.cuda.synchronize()
+    want_out, want_k = run.out.clone(), run.cache.k.clone()
+    run.rewind()
+    run.cache.k[:, :, :, w.ctx_blocks - 1].zero_()   # the row the step appends
+    run.out.zero_()
+    run.step_host()
+    torch.cuda.synchronize()
+    assert run.status.item() == 0 and (run.cache.len == w.ctx_blocks).all()
+    assert torch.equal(run.out, want_out) and torch.equal(run.cache.k, want_k)
+    assert torch.equal(run._host["out"], want_out.cpu())   # and the host copy of the result
+
+
 def test_token_decode_full_size_two_blocks(bt):
     """BASELINE configs[2]: 4096 sequences, 12 layers, local cache 1 prefix + up to L_B rows; two
     blocks of consecutive token steps, lengths against the integer schedule model at full size."""
