@@ -705,9 +705,11 @@ block_prefill_tc_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_c
                 mbar_arrive(bar(B_P1FULL + x));
                 PF_EVS(5);
             }
+            // From here to the named barrier below no thread leaves early: a thread whose wait ran out (ok ==
+            // false; later waits then give up soon, the abort flag being up) still stages its row and meets the others, and the
+            // barrier tells all 128 whether any of them failed, so that they give up at the same item.
             if (ok) ok = mbar_wait(bar(B_OFULL + x), o_count & 1, abort_flag, p.dev_status);
             ++o_count;
-            if (!ok) break;
             PF_EVS(6);
             tc_fence_after();
             const float inv = l > 0.f ? 1.f / l : 0.f;
@@ -736,7 +738,16 @@ block_prefill_tc_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_c
             tc_fence_before();
             asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
             PF_EVS(7);
-            asm volatile("barrier.sync.aligned %0, 128;" ::"r"(1 + x) : "memory");  // the warpgroup's 128 rows are staged
+            uint32_t any_failed;  // the warpgroup's 128 rows are staged; did a wait run out in any of its threads?
+            asm volatile(
+                "{\n\t.reg .pred p, q;\n\t"
+                "setp.ne.u32 q, %2, 0;\n\t"
+                "bar.red.or.pred p, %1, 128, q;\n\t"
+                "selp.u32 %0, 1, 0, p;\n\t}"
+                : "=r"(any_failed)
+                : "r"(1 + x), "r"(ok ? 0u : 1u)
+                : "memory");
+            if (any_failed) break;
             if (wq == 0 && lane == 0) {
                 for (int bx = 0; bx < NB; ++bx)
                     tma_store_3d(&mapO, sV + stage_o * TILE_BYTES + bx * kBoxBytes, bx * 64, qt * BM, it.bh);
