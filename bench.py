@@ -278,9 +278,9 @@ def run_gpu(args):
         for _ in range(3):
             run.replay_timed()
         torch.cuda.synchronize()
-        clocks = sampler.stop()
         kern_events = run.graph_events
         ms_e2e = timed(run.step_host, run.rewind, args.steps, args.warmup)
+        clocks = sampler.stop()  # sampled over the device-resident, the attention-only and the host-buffer runs
         h2d, d2h = run.host_bytes_per_step()
         alg_bytes = traffic.block_decode_layer_bytes(w.batch, w.heads, w.head_dim, w.ctx_blocks, with_append=False)
         dom = "block_decode_ring_kernel"
