@@ -112,22 +112,30 @@ dist_env = replicas.dist_env
 
 # ------------------------------------------------------------------------------------------ CPU oracle legs
 
-def oracle_block_decode_sample(w, n_seq, seed=None):
-    """Time the oracle on n_seq sequences of one layer of the block-decode step; returns
-    (seconds, sequences, layers) of the sample."""
-    import oracle
-    seed = w.seed if seed is None else seed
-    B, H, hd, N = n_seq, w.heads, w.head_dim, w.max_blocks
-    c = oracle.Cache(B, H, N, hd)
-    c.k[...] = gen.normal_bf16_bits(seed, 0, c.k.shape)
-    c.v[...] = gen.normal_bf16_bits(seed, 1, c.v.shape)
-    c.len[...] = w.ctx_blocks - 1
-    q, k, v = (gen.normal_bf16_bits(seed, 2 + i, (B, H, 1, hd)) for i in range(3))
-    oracle.lib()
-    t0 = time.perf_counter()
-    oracle.kv_append(c, k, v)
-    oracle.block_decode_attn(c, np.ascontiguousarray(q[:, :, 0]))
-    return time.perf_counter() - t0, n_seq, 1
+class OracleBlockDecodeSample:
+    """The oracle on n_seq sequences of one layer of the block-decode step.  The inputs are drawn once;
+    every step() puts the lengths back and times append + attention."""
+
+    def __init__(self, w, n_seq, seed=None):
+        import oracle
+        seed = w.seed if seed is None else seed
+        self.w, self.n_seq = w, n_seq
+        B, H, hd, N = n_seq, w.heads, w.head_dim, w.max_blocks
+        self.c = oracle.Cache(B, H, N, hd)
+        self.c.k[...] = gen.normal_bf16_bits(seed, 0, self.c.k.shape)
+        self.c.v[...] = gen.normal_bf16_bits(seed, 1, self.c.v.shape)
+        self.q, self.k, self.v = (gen.normal_bf16_bits(seed, 2 + i, (B, H, 1, hd)) for i in range(3))
+        self.q0 = np.ascontiguousarray(self.q[:, :, 0])
+        oracle.lib()
+
+    def step(self):
+        """Returns the seconds the oracle took for one sample."""
+        import oracle
+        self.c.len[...] = self.w.ctx_blocks - 1
+        t0 = time.perf_counter()
+        oracle.kv_append(self.c, self.k, self.v)
+        oracle.block_decode_attn(self.c, self.q0)
+        return time.perf_counter() - t0
 
 
 def cpu_baseline_block_decode(w, run):
@@ -164,12 +172,10 @@ def run_reference(args):
         return 0
     w = configs.BY_NAME[args.workload]
     n_seq = 64
+    sample_run = OracleBlockDecodeSample(w, n_seq)
     for _ in range(max(1, min(args.warmup, 2))):
-        oracle_block_decode_sample(w, n_seq)
-    times = []
-    for _ in range(args.steps):
-        secs, ns, nl = oracle_block_decode_sample(w, n_seq)
-        times.append(secs)
+        sample_run.step()
+    times = [sample_run.step() for _ in range(args.steps)]
     scale = (w.batch / n_seq) * w.n_layers
     step_s = statistics.mean(times) * scale
     tokens = w.batch * w.block_len
