@@ -92,11 +92,20 @@ typedef struct bt_local_cache {
 int bt_version(void);
 const char* bt_status_string(bt_status s);
 
-/* Number of ways bt_block_decode_attn will split each (sequence, head) row range for this
- * config (>= 1), and the workspace it then needs: splits * B * H * (hd + 4) floats when
- * splits > 1, else 0.  Both return 0 on an invalid config.                              */
+/* Number of ways the block-decoder decode kernel splits each (sequence, head) row range for this
+ * config (>= 1), and the size of the workspace of the decode calls: splits * B * H * (hd + 4) floats
+ * of per-split partial results when splits > 1, then B * H + B int32 arrival counters.  Both
+ * return 0 on an invalid config.
+ *
+ * bt_workspace_init zeroes the counters (asynchronously, on the stream).  A workspace must be
+ * initialised once - by this call, or by zero-filling it - before its first use; every decode
+ * call leaves the counters at zero again, so it is never needed a second time, except after a
+ * call that raised BT_DEV_TIMEOUT (which may leave counts behind).  The partial results need no
+ * initialisation.  A workspace serves one call at a time: calls that can overlap on the GPU need
+ * one each.                                                                                   */
 int bt_decode_splits(const bt_config* cfg);
 size_t bt_workspace_bytes(const bt_config* cfg);
+bt_status bt_workspace_init(const bt_config* cfg, void* workspace, size_t workspace_bytes, void* stream);
 
 /*
  * Block-decoder KV append (sections 2.1 and 2.3: the K,V of every processed block are cached,
@@ -114,12 +123,29 @@ bt_status bt_block_kv_append(const bt_config* cfg, bt_block_cache* cache, int la
  *   out[b,h,:] = sum_j softmax_j(scale * q[b,h,:] . K[b,h,j,:]) * V[b,h,j,:],  j < len[b],
  * i.e. the query of the newest block attends to every cached block including its own row
  * len[b]-1.  q, out: [B][H][hd].  len[b] == 0 gives zeros and BT_DEV_EMPTY.
- * workspace: device scratch of at least bt_workspace_bytes(cfg) bytes (may be NULL when that
- * is 0); it holds the per-split partial results and needs no initialisation.
+ * workspace: device scratch of at least bt_workspace_bytes(cfg) bytes, initialised as described
+ * there (may be NULL when bt_decode_splits(cfg) is 1: an unsplit row range needs none).  With a
+ * split range each part writes its partial result there and the part that finishes last combines
+ * them by the log-sum-exp rule, inside the same launch.
  */
 bt_status bt_block_decode_attn(const bt_config* cfg, const bt_block_cache* cache, int layer,
                                const void* q, void* out, void* workspace, size_t workspace_bytes,
                                uint32_t* dev_status, void* stream);
+
+/*
+ * One block-decoder decode step of a layer in a single launch (section 2.3: per generated block,
+ * the block's K,V are cached and its query attends to every cached block including itself):
+ * exactly bt_block_kv_append with n_new = 1 followed by bt_block_decode_attn.  For each sequence
+ * b with len[b] < N_max: row len[b] of every head receives k_new / v_new [B][H][hd], the query
+ * attends to rows 0 .. len[b] (the new row comes from k_new / v_new, the rest from the cache), and
+ * len[b] += 1.  A sequence whose cache is full is left as it is, attended over its N_max rows, and
+ * BT_DEV_OVERFLOW is raised.  workspace: required (never NULL), as for bt_block_decode_attn.
+ * The cache rows, the lengths and out are all written by this one launch; k_new, v_new and q must
+ * not alias them.
+ */
+bt_status bt_block_decode_step(const bt_config* cfg, bt_block_cache* cache, int layer, const void* q,
+                               const void* k_new, const void* v_new, void* out, void* workspace,
+                               size_t workspace_bytes, uint32_t* dev_status, void* stream);
 
 /*
  * bt_block_decode_attn for callers that cannot supply a workspace.  (The paper has no
@@ -136,8 +162,9 @@ bt_status bt_block_decode_attn(const bt_config* cfg, const bt_block_cache* cache
  *   - The first call on each device whose config splits the row range looks up the array's
  *     address on that device (the device must be current, as for every call here, and own the
  *     buffers passed in).  Make that first call outside any stream capture.
- *   - All calls on one device share the array.  It needs no clearing (every partial is written
- *     before it is read within one call, so what an earlier call left behind is never seen), but
+ *   - All calls on one device share the array, whatever their config.  The caller never clears
+ *     it: each call zeroes its own arrival counters first (a memset on the stream), and every
+ *     partial is written before it is read within one call.  But
  *     two calls that can overlap on the GPU (different streams, no dependency) race on it:
  *     order them, or give one of them bt_block_decode_attn with its own workspace.
  * Other arguments, results and errors are those of bt_block_decode_attn.
@@ -198,10 +225,10 @@ bt_status bt_block_prefill_attn(const bt_config* cfg, const void* q, const void*
                                 void* stream);
 
 /*
- * One block-decoder decode step of one layer driven from HOST buffers (the same operations as
- * bt_block_kv_append followed by bt_block_decode_attn, section 2.3): q_host, k_new_host,
+ * One block-decoder decode step of one layer driven from HOST buffers (bt_block_decode_step with
+ * the copies around it, section 2.3): q_host, k_new_host,
  * v_new_host [B][H][hd] bf16 are copied to the caller's device staging buffers q_dev, k_dev,
- * v_dev, the row is appended, attention runs, and out_dev is copied to out_host [B][H][hd].
+ * v_dev, the row is appended and attended over in one launch, and out_dev is copied to out_host [B][H][hd].
  * Host buffers should be pinned; all copies are asynchronous on `stream`.
  */
 bt_status bt_block_decode_step_host(const bt_config* cfg, bt_block_cache* cache, int layer,

@@ -21,6 +21,7 @@ EXPORTS = [
     "bt_version", "bt_status_string", "bt_decode_splits", "bt_workspace_bytes", "bt_block_kv_append",
     "bt_block_decode_attn", "bt_local_kv_reset", "bt_local_kv_append", "bt_token_decode_attn",
     "bt_block_prefill_attn", "bt_block_decode_step_host", "bt_block_decode_attn_noalloc",
+    "bt_workspace_init", "bt_block_decode_step",
 ]
 
 
@@ -61,6 +62,8 @@ def _load() -> ctypes.CDLL:
     lib.bt_workspace_bytes.argtypes = [cfgp]
     lib.bt_block_kv_append.argtypes = [cfgp, ctypes.POINTER(bt_block_cache), i32, vp, vp, i32, vp, vp]
     lib.bt_block_decode_attn.argtypes = [cfgp, ctypes.POINTER(bt_block_cache), i32, vp, vp, vp, u64, vp, vp]
+    lib.bt_workspace_init.argtypes = [cfgp, vp, u64, vp]
+    lib.bt_block_decode_step.argtypes = [cfgp, ctypes.POINTER(bt_block_cache), i32, vp, vp, vp, vp, vp, u64, vp, vp]
     lib.bt_local_kv_reset.argtypes = [cfgp, ctypes.POINTER(bt_local_cache), i32, vp, vp]
     lib.bt_local_kv_append.argtypes = [cfgp, ctypes.POINTER(bt_local_cache), i32, vp, vp, i32, vp, vp]
     lib.bt_token_decode_attn.argtypes = [cfgp, ctypes.POINTER(bt_local_cache), i32, vp, vp, vp, i32, i32, vp, vp, vp, vp]
@@ -144,9 +147,17 @@ def bt_workspace_bytes(cfg) -> int:
     return _lib.bt_workspace_bytes(ctypes.byref(cfg))
 
 
+def bt_workspace_init(cfg, workspace, stream=None):
+    _check(_lib.bt_workspace_init(ctypes.byref(cfg), _ptr(workspace), workspace.numel() * workspace.element_size(),
+                                  _stream(stream)), "bt_workspace_init")
+
+
 def alloc_workspace(cfg, device="cuda"):
+    """A workspace for the decode calls of this config, initialised (counters zeroed) and ready."""
     n = bt_workspace_bytes(cfg)
-    return torch.empty(max(n, 4) // 4, dtype=torch.float32, device=device)
+    ws = torch.empty((max(n, 4) + 3) // 4, dtype=torch.float32, device=device)
+    bt_workspace_init(cfg, ws)
+    return ws
 
 
 def bt_block_kv_append(cfg, cache: BlockCache, layer, k_new, v_new, n_new=None, dev_status=None, stream=None):
@@ -160,6 +171,13 @@ def bt_block_decode_attn(cfg, cache: BlockCache, layer, q, out, workspace=None, 
     _check(_lib.bt_block_decode_attn(ctypes.byref(cfg), ctypes.byref(cache.c), layer, _ptr(q), _ptr(out),
                                      _ptr(workspace), ws_bytes, _ptr(dev_status), _stream(stream)),
            "bt_block_decode_attn")
+
+
+def bt_block_decode_step(cfg, cache: BlockCache, layer, q, k_new, v_new, out, workspace, dev_status=None, stream=None):
+    """Append the new block's row and attend over the cache including it, in one launch."""
+    _check(_lib.bt_block_decode_step(ctypes.byref(cfg), ctypes.byref(cache.c), layer, _ptr(q), _ptr(k_new), _ptr(v_new),
+                                     _ptr(out), _ptr(workspace), workspace.numel() * workspace.element_size(),
+                                     _ptr(dev_status), _stream(stream)), "bt_block_decode_step")
 
 
 BT_STATIC_WORKSPACE_BYTES = 2 << 20

@@ -105,12 +105,28 @@ int bt_decode_splits(const bt_config* cfg)
     return choose_splits(cfg);
 }
 
+// Workspace layout: the split partials ([B*H][splits][hd+4] floats, absent when the row range is not
+// split), then the arrival counters ([B*H] + [B] int32).
+static size_t partial_bytes(const bt_config* cfg)
+{
+    const int s = choose_splits(cfg);
+    return s <= 1 ? 0 : (size_t)s * cfg->batch * cfg->heads * (cfg->head_dim + 4) * sizeof(float);
+}
+static size_t counter_bytes(const bt_config* cfg) { return ((size_t)cfg->batch * cfg->heads + cfg->batch) * sizeof(int32_t); }
+
 size_t bt_workspace_bytes(const bt_config* cfg)
 {
     if (check_config(cfg, 0) != BT_OK) return 0;
-    const int s = choose_splits(cfg);
-    if (s <= 1) return 0;
-    return (size_t)s * cfg->batch * cfg->heads * (cfg->head_dim + 4) * sizeof(float);
+    return partial_bytes(cfg) + counter_bytes(cfg);
+}
+
+bt_status bt_workspace_init(const bt_config* cfg, void* workspace, size_t workspace_bytes, void* stream)
+{
+    bt_status st = check_config(cfg, 0);
+    if (st != BT_OK) return st;
+    if (!workspace) return BT_ERR_NULL;
+    if (workspace_bytes < bt_workspace_bytes(cfg)) return BT_ERR_WORKSPACE;
+    return cuda_status(cudaMemsetAsync((char*)workspace + partial_bytes(cfg), 0, counter_bytes(cfg), (cudaStream_t)stream));
 }
 
 bt_status bt_block_kv_append(const bt_config* cfg, bt_block_cache* cache, int layer, const void* k_new,
@@ -125,15 +141,14 @@ bt_status bt_block_kv_append(const bt_config* cfg, bt_block_cache* cache, int la
                                             k_new, v_new, n_new, dev_status, (cudaStream_t)stream));
 }
 
-bt_status bt_block_decode_attn(const bt_config* cfg, const bt_block_cache* cache, int layer, const void* q,
-                               void* out, void* workspace, size_t workspace_bytes, uint32_t* dev_status,
-                               void* stream)
+// append (optional) + attention in one launch
+static bt_status decode_launch(const bt_config* cfg, bt_block_cache* cache, int layer, const void* q, const void* k_new,
+                               const void* v_new, void* out, void* workspace, size_t workspace_bytes,
+                               uint32_t* dev_status, void* stream)
 {
-    bt_status st = check_config(cfg, layer);
-    if (st != BT_OK) return st;
-    if (!cache || !cache->k || !cache->v || !cache->len || !q || !out) return BT_ERR_NULL;
-    const size_t need = bt_workspace_bytes(cfg);
-    if (need && (!workspace || workspace_bytes < need)) return BT_ERR_WORKSPACE;
+    const int splits = choose_splits(cfg);
+    const bool need_ws = splits > 1 || k_new != nullptr;
+    if (need_ws && (!workspace || workspace_bytes < bt_workspace_bytes(cfg))) return BT_ERR_WORKSPACE;
     bt::CacheView v = block_view(cfg, cache, layer);
     bt::DecodeArgs a;
     a.q = q;
@@ -142,14 +157,39 @@ bt_status bt_block_decode_attn(const bt_config* cfg, const bt_block_cache* cache
     a.len = v.len;
     a.out = out;
     a.ws = (float*)workspace;
+    a.counters = need_ws ? (int32_t*)((char*)workspace + partial_bytes(cfg)) : nullptr;
+    a.k_new = k_new;
+    a.v_new = v_new;
     a.dev_status = dev_status;
     a.B = cfg->batch;
     a.H = cfg->heads;
     a.hd = cfg->head_dim;
     a.n_max = cfg->max_blocks;
-    a.splits = choose_splits(cfg);
+    a.splits = splits;
     a.scale_log2 = scale_log2(cfg);
     return cuda_status(bt::launch_block_decode(a, (cudaStream_t)stream));
+}
+
+bt_status bt_block_decode_attn(const bt_config* cfg, const bt_block_cache* cache, int layer, const void* q,
+                               void* out, void* workspace, size_t workspace_bytes, uint32_t* dev_status,
+                               void* stream)
+{
+    bt_status st = check_config(cfg, layer);
+    if (st != BT_OK) return st;
+    if (!cache || !cache->k || !cache->v || !cache->len || !q || !out) return BT_ERR_NULL;
+    // without a row to append the kernel only reads the cache
+    return decode_launch(cfg, const_cast<bt_block_cache*>(cache), layer, q, nullptr, nullptr, out, workspace,
+                         workspace_bytes, dev_status, stream);
+}
+
+bt_status bt_block_decode_step(const bt_config* cfg, bt_block_cache* cache, int layer, const void* q,
+                               const void* k_new, const void* v_new, void* out, void* workspace,
+                               size_t workspace_bytes, uint32_t* dev_status, void* stream)
+{
+    bt_status st = check_config(cfg, layer);
+    if (st != BT_OK) return st;
+    if (!cache || !cache->k || !cache->v || !cache->len || !q || !k_new || !v_new || !out) return BT_ERR_NULL;
+    return decode_launch(cfg, cache, layer, q, k_new, v_new, out, workspace, workspace_bytes, dev_status, stream);
 }
 
 bt_status bt_local_kv_reset(const bt_config* cfg, bt_local_cache* cache, int layer, const uint8_t* seq_mask,
@@ -241,9 +281,7 @@ bt_status bt_block_decode_step_host(const bt_config* cfg, bt_block_cache* cache,
     if (cudaMemcpyAsync(k_dev, k_new_host, bytes, cudaMemcpyHostToDevice, s) != cudaSuccess) return BT_ERR_CUDA;
     if (cudaMemcpyAsync(v_dev, v_new_host, bytes, cudaMemcpyHostToDevice, s) != cudaSuccess) return BT_ERR_CUDA;
     if (cudaMemcpyAsync(q_dev, q_host, bytes, cudaMemcpyHostToDevice, s) != cudaSuccess) return BT_ERR_CUDA;
-    st = bt_block_kv_append(cfg, cache, layer, k_dev, v_dev, 1, dev_status, stream);
-    if (st != BT_OK) return st;
-    st = bt_block_decode_attn(cfg, cache, layer, q_dev, out_dev, workspace, workspace_bytes, dev_status, stream);
+    st = bt_block_decode_step(cfg, cache, layer, q_dev, k_dev, v_dev, out_dev, workspace, workspace_bytes, dev_status, stream);
     if (st != BT_OK) return st;
     if (cudaMemcpyAsync(out_host, out_dev, bytes, cudaMemcpyDeviceToHost, s) != cudaSuccess) return BT_ERR_CUDA;
     return BT_OK;

@@ -10,6 +10,14 @@
 // lane group of hd/8 lanes owns a row: 128-bit shared-memory reads, fp32 dot product reduced by
 // shuffles, online softmax in the log2 domain per lane; row groups merge by shuffles at the end of
 // the item.  Every wait on a copy is bounded and raises BT_DEV_TIMEOUT when it runs out.
+//
+// Two things ride along so that a decode step is one launch per layer.  (1) Split row ranges: every
+// item writes its normalised partial and log2-sum-exp, then counts itself in; the item that arrives
+// last for a (sequence, head) folds all partials by the log-sum-exp rule and writes the output, so
+// no merge launch follows.  (2) Fused append: when a new row is passed in, the item that owns the
+// last row takes it from the caller's buffer (and stores it into the cache) instead of streaming
+// it; the sequence's length is raised by the item that is last to finish with that sequence, once
+// every item has read the old one.  Both counters return to zero before the kernel ends.
 #include "bt_common.cuh"
 #include "bt_kernels.h"
 
@@ -92,9 +100,11 @@ __device__ __forceinline__ uint4 lds128(uint32_t addr)
     return r;
 }
 
-// Row range of one work item.
+// Row range of one work item.  n counts the appended row when there is one; rows [r0, c1) come from
+// the cache, and row n-1 from the caller's buffer when new_row is set.
 struct Work {
-    int bh, sp, b, n, r0, r1;
+    int bh, sp, b, n, r0, c1;
+    bool new_row, overflow;
 };
 __device__ __forceinline__ Work decode_work(int item, const DecodeArgs& a)
 {
@@ -104,16 +114,22 @@ __device__ __forceinline__ Work decode_work(int item, const DecodeArgs& a)
     w.b = w.bh / a.H;
     int n = a.len[w.b];
     n = n < 0 ? 0 : (n > a.n_max ? a.n_max : n);
+    const bool append = a.k_new != nullptr && n < a.n_max;  // a full cache takes no row: flagged, attended as it is
+    w.overflow = a.k_new != nullptr && !append;
+    n += append ? 1 : 0;
     w.n = n;
     const int per = (n + a.splits - 1) / a.splits;
     w.r0 = min(n, w.sp * per);
-    w.r1 = min(n, w.r0 + per);
+    const int r1 = min(n, w.r0 + per);
+    w.new_row = append && r1 == n && w.r0 < n;   // exactly one split ends at row n-1
+    w.c1 = w.new_row ? r1 - 1 : r1;
     return w;
 }
 
 // grid: one CTA per SM (fewer when there are fewer items than warps).  splits == 1 writes bf16
-// output directly; otherwise each item writes its normalised partial (hd floats) and its
-// log2-sum-exp to the workspace and decode_merge_kernel combines them.
+// output directly; otherwise each item writes its normalised partial (hd floats, then its
+// log2-sum-exp; hd+4 floats apart so that every partial is 16-byte aligned) to the workspace and the
+// last one to arrive combines them.
 template <int HD>
 __global__ void __launch_bounds__(kThreads, 1) block_decode_ring_kernel(DecodeArgs a)
 {
@@ -138,8 +154,8 @@ __global__ void __launch_bounds__(kThreads, 1) block_decode_ring_kernel(DecodeAr
     const int n_items = a.B * a.H * a.splits;
     const int stride = kWarps * gridDim.x;
     const int first = warp * gridDim.x + blockIdx.x;   // neighbouring items go to different SMs
-    const bf16* Kall = reinterpret_cast<const bf16*>(a.k);
-    const bf16* Vall = reinterpret_cast<const bf16*>(a.v);
+    bf16* Kall = reinterpret_cast<bf16*>(a.k);
+    bf16* Vall = reinterpret_cast<bf16*>(a.v);
     // While the kernel before this one drains, warm L2 with the first ring-full of this warp's first
     // item (rows 0.. of its slab, whatever its length turns out to be: the rows exist either way), its
     // length and its query.  A prefetch returns nothing to the thread, so it is safe ahead of the wait.
@@ -163,7 +179,7 @@ __global__ void __launch_bounds__(kThreads, 1) block_decode_ring_kernel(DecodeAr
     auto p_seek = [&]() {  // move to the next item that has rows
         while (p_item < n_items) {
             pw = decode_work(p_item, a);
-            p_nchunks = (pw.r1 - pw.r0 + ROWS - 1) / ROWS;
+            p_nchunks = (pw.c1 - pw.r0 + ROWS - 1) / ROWS;
             if (p_nchunks > 0) {
                 p_c = 0;
                 return;
@@ -175,7 +191,7 @@ __global__ void __launch_bounds__(kThreads, 1) block_decode_ring_kernel(DecodeAr
     auto issue_one = [&]() {
         if (p_item >= n_items) return;
         const int row = pw.r0 + p_c * ROWS;
-        const uint32_t bytes = (uint32_t)min(ROWS, pw.r1 - row) * G::ROW_BYTES;
+        const uint32_t bytes = (uint32_t)min(ROWS, pw.c1 - row) * G::ROW_BYTES;
         const uint32_t st = issued % kStages;
         if (lane == 0) {
             const uint32_t bar = bar0 + 8 * st, dst = ring0 + st * G::STAGE_BYTES;
@@ -200,6 +216,17 @@ __global__ void __launch_bounds__(kThreads, 1) block_decode_ring_kernel(DecodeAr
     if (first < n_items) q_next = ld_plain(Qall + (size_t)(first / a.splits) * HD + sub * 8);
     for (int item = first; alive && item < n_items; item += stride) {
         const Work w = decode_work(item, a);
+        // Fused append: the sequence's length goes up once all of its H * splits items have read the old
+        // one.  An item counts itself in as soon as its own read has returned (the increment is computed
+        // from the value read, so the count cannot be issued before that) and looks at the result only
+        // when it is done, a whole item later: nothing ever waits for the round trip.  Whoever counted in
+        // last raises the length.  (This warp's look-ahead read of the same length came even earlier.)
+        int seq_arrival = -1;
+        if (a.k_new != nullptr && lane == 0) {
+            int one;
+            asm volatile("and.b32 %0, %1, 0;\n\tadd.s32 %0, %0, 1;" : "=r"(one) : "r"(w.n));
+            seq_arrival = atomicAdd(a.counters + (size_t)a.B * a.H + w.b, one);
+        }
         float qf[8];
         {
             const uint4 qr = q_next;
@@ -208,16 +235,22 @@ __global__ void __launch_bounds__(kThreads, 1) block_decode_ring_kernel(DecodeAr
 #pragma unroll
             for (int i = 0; i < 8; ++i) qf[i] *= a.scale_log2;
         }
+        // the appended row, when this item owns it: fetched now, used after the cached rows
+        uint4 kn = make_uint4(0, 0, 0, 0), vn = kn;
+        if (w.new_row) {
+            kn = ld_plain(reinterpret_cast<const bf16*>(a.k_new) + (size_t)w.bh * HD + sub * 8);
+            vn = ld_plain(reinterpret_cast<const bf16*>(a.v_new) + (size_t)w.bh * HD + sub * 8);
+        }
         SoftmaxState st;
         st.init();
-        const int nchunks = (w.r1 - w.r0 + ROWS - 1) / ROWS;
+        const int nchunks = (w.c1 - w.r0 + ROWS - 1) / ROWS;
         for (int c = 0; c < nchunks; ++c) {
             const uint32_t sidx = consumed % kStages;
             if (!mbar_wait_bounded(bar0 + 8 * sidx, (consumed / kStages) & 1)) {
                 alive = false;
                 break;
             }
-            const int nvalid = min(ROWS, w.r1 - (w.r0 + c * ROWS));
+            const int nvalid = min(ROWS, w.c1 - (w.r0 + c * ROWS));
             const uint32_t ks = ring0 + sidx * G::STAGE_BYTES + rg * G::ROW_BYTES + sub * 16;
             const uint32_t vs = ks + G::CHUNK_BYTES;
             uint4 kr[kUnroll], vr[kUnroll];
@@ -274,30 +307,83 @@ __global__ void __launch_bounds__(kThreads, 1) block_decode_ring_kernel(DecodeAr
             }
         }
         if (!alive) break;
-        // merge the RPW row groups of the warp
+        if (w.new_row) {  // warp-uniform.  Row n-1 = the new row: scored from registers, stored into the cache
+            const float sn = row_sum<LPR>(dot8(qf, kn));
+            if (rg == 0) {
+                const float mn = fmaxf(st.m, sn);
+                const float cf = ex2(st.m - mn), pn = ex2(sn - mn);
+                st.l = st.l * cf + pn;
 #pragma unroll
-        for (int off = LPR; off < 32; off <<= 1) {
-            const float m2 = __shfl_xor_sync(0xffffffffu, st.m, off);
-            const float l2 = __shfl_xor_sync(0xffffffffu, st.l, off);
-            float a2[8];
-#pragma unroll
-            for (int i = 0; i < 8; ++i) a2[i] = __shfl_xor_sync(0xffffffffu, st.acc[i], off);
-            st.merge(m2, l2, a2);
+                for (int i = 0; i < 8; ++i) st.acc[i] *= cf;
+                fma8(st.acc, pn, vn);
+                st.m = mn;
+                const size_t off = ((size_t)w.bh * a.n_max + (w.n - 1)) * HD + sub * 8;
+                *reinterpret_cast<uint4*>(Kall + off) = kn;
+                *reinterpret_cast<uint4*>(Vall + off) = vn;
+            }
         }
-        if (rg == 0) {
+        // merge the RPW row groups of the warp
+        auto merge_row_groups = [&]() {
+#pragma unroll
+            for (int off = LPR; off < 32; off <<= 1) {
+                const float m2 = __shfl_xor_sync(0xffffffffu, st.m, off);
+                const float l2 = __shfl_xor_sync(0xffffffffu, st.l, off);
+                float a2[8];
+#pragma unroll
+                for (int i = 0; i < 8; ++i) a2[i] = __shfl_xor_sync(0xffffffffu, st.acc[i], off);
+                st.merge(m2, l2, a2);
+            }
+        };
+        auto write_out = [&]() {  // lanes of row group 0: normalised bf16 output row
             float o[8];
             const float inv = st.l > 0.f ? 1.f / st.l : 0.f;
 #pragma unroll
             for (int i = 0; i < 8; ++i) o[i] = st.acc[i] * inv;
-            if (a.splits == 1) {
-                *reinterpret_cast<uint4*>(reinterpret_cast<bf16*>(a.out) + (size_t)w.bh * HD + sub * 8) = pack8(o);
-            } else {
+            *reinterpret_cast<uint4*>(reinterpret_cast<bf16*>(a.out) + (size_t)w.bh * HD + sub * 8) = pack8(o);
+        };
+        merge_row_groups();
+        if (a.splits == 1) {
+            if (rg == 0) write_out();
+        } else {
+            if (rg == 0) {
+                float o[8];
+                const float inv = st.l > 0.f ? 1.f / st.l : 0.f;
+#pragma unroll
+                for (int i = 0; i < 8; ++i) o[i] = st.acc[i] * inv;
                 float* ws = a.ws + ((size_t)w.bh * a.splits + w.sp) * (HD + 4);
                 *reinterpret_cast<float4*>(ws + sub * 8) = make_float4(o[0], o[1], o[2], o[3]);
                 *reinterpret_cast<float4*>(ws + sub * 8 + 4) = make_float4(o[4], o[5], o[6], o[7]);
                 if (sub == 0) ws[HD] = st.l > 0.f ? st.m + log2f(st.l) : kNegInf;
+                __threadfence();  // the partial is visible before this item counts itself in
             }
-            if (sub == 0 && w.sp == 0 && w.n == 0 && (w.bh % a.H) == 0) raise_status(a.dev_status, BT_DEV_EMPTY);
+            __syncwarp();
+            int last = 0;
+            if (lane == 0) last = atomicAdd(a.counters + w.bh, 1) == a.splits - 1;
+            last = __shfl_sync(0xffffffffu, last, 0);
+            if (last) {  // every split of (b,h) has written: fold the partials (normalised, weight 2^lse each)
+                __threadfence();
+                st.init();
+                for (int s2 = rg; s2 < a.splits; s2 += RPW) {
+                    const float* ws = a.ws + ((size_t)w.bh * a.splits + s2) * (HD + 4);
+                    const float lse = __ldcg(ws + HD);
+                    const float4 x = __ldcg(reinterpret_cast<const float4*>(ws + sub * 8));
+                    const float4 y = __ldcg(reinterpret_cast<const float4*>(ws + sub * 8 + 4));
+                    const float a2[8] = {x.x, x.y, x.z, x.w, y.x, y.y, y.z, y.w};
+                    st.merge(lse, 1.f, a2);
+                }
+                merge_row_groups();
+                if (rg == 0) write_out();
+                if (lane == 0) a.counters[w.bh] = 0;
+            }
+        }
+        if (w.sp == 0 && (w.bh % a.H) == 0 && lane == 0) {
+            if (w.n == 0) raise_status(a.dev_status, BT_DEV_EMPTY);
+            if (w.overflow) raise_status(a.dev_status, BT_DEV_OVERFLOW);
+        }
+        if (seq_arrival == a.H * a.splits - 1) {
+            // this item was the last of its sequence to read the old length (lane 0 only): raise it
+            if (!w.overflow) a.len[w.b] = w.n;
+            a.counters[(size_t)a.B * a.H + w.b] = 0;
         }
     }
     if (!alive) {
@@ -335,7 +421,7 @@ static cudaError_t launch_t(const DecodeArgs& a, cudaStream_t stream)
 
 }  // namespace ring
 
-cudaError_t launch_block_decode_ring(const DecodeArgs& a, cudaStream_t stream)
+cudaError_t launch_block_decode(const DecodeArgs& a, cudaStream_t stream)
 {
     return a.hd == 64 ? ring::launch_t<64>(a, stream) : ring::launch_t<128>(a, stream);
 }

@@ -24,18 +24,23 @@ cudaError_t launch_len_reset(int32_t* len, int B, const uint8_t* mask, cudaStrea
 
 struct DecodeArgs {
     const void* q;       // [B][H][hd]
-    const void* k;       // layer base, [B][H][N_max][hd]
-    const void* v;
-    const int32_t* len;  // [B]
+    void* k;             // layer base, [B][H][N_max][hd] (written only by the fused append)
+    void* v;
+    int32_t* len;        // [B] (written only by the fused append)
     void* out;           // [B][H][hd]
     float* ws;           // [B*H][splits][hd+4] when splits > 1
+    // arrival counters, zero on entry and left zero: [B*H] (splits of a (b,h) that have written their
+    // partial) then [B] (items of a sequence that are done with its length).  Needed when splits > 1 or
+    // when a row is appended; may be NULL otherwise.
+    int32_t* counters;
+    const void* k_new;   // fused append: [B][H][hd], the row that becomes row len[b]; NULL = attention only
+    const void* v_new;
     uint32_t* dev_status;
     int B, H, hd, n_max, splits;
     float scale_log2;    // softmax scale * log2(e)
 };
+// The streaming kernel: per-item results, or per-split partials merged by the split that finishes last.
 cudaError_t launch_block_decode(const DecodeArgs& a, cudaStream_t stream);
-// The streaming kernel alone (per-item results or per-split partials; no merge pass).
-cudaError_t launch_block_decode_ring(const DecodeArgs& a, cudaStream_t stream);
 
 struct TokenArgs {
     void* kv;            // layer base, [B][H][C][2][hd]

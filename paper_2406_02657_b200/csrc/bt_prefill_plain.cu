@@ -1,7 +1,6 @@
-// Block-decoder decode attention, second half (paper section 2.3; appendix E.2): the streaming kernel
-// lives in bt_decode_ring.cu; here are the merge of the per-split partial results by the log-sum-exp
-// rule, and the plain CUDA-core prefill kernel (one query block per CTA over rows 0..t, 128-bit
-// read-once loads, online softmax per lane) that serves shapes the tensor-core kernel does not take.
+// Block-decoder prefill on the CUDA cores (paper section 2.3: the block decoder is causal over blocks):
+// one query block per CTA over rows 0..t, 128-bit read-once loads, online softmax per lane.  It serves
+// the shapes the tensor-core kernel does not take, and as its cross-check.
 #include "bt_common.cuh"
 #include "bt_kernels.h"
 
@@ -10,10 +9,6 @@ namespace bt {
 constexpr int kDecodeWarps = 4;
 constexpr int kDecodeThreads = kDecodeWarps * 32;
 constexpr int kUnroll = 8;  // independent K (and V) loads in flight per lane
-// floats per split partial in the workspace: hd outputs + log2-sum-exp, padded so that every
-// partial starts on a 16-byte boundary (the outputs are stored as float4)
-template <int HD>
-constexpr int kPartStride = HD + 4;
 
 // Attention of one query over rows [r0, r1) of one (b,h) slab, by one CTA of kDecodeWarps
 // warps.  On return, threads 0..LPR-1 of warp 0 hold the merged state for their 8 dims
@@ -105,53 +100,6 @@ __device__ __forceinline__ void attend_range(const bf16* __restrict__ qrow, cons
             st.merge(w[HD], w[HD + 1], a2);
         }
     }
-}
-
-// Combine the per-split partials: out = sum_s w_s o_s with w_s = 2^(lse_s - max) / sum.
-// One lane group of LPR threads per (b,h).
-template <int HD>
-__global__ void __launch_bounds__(128) decode_merge_kernel(DecodeArgs a)
-{
-    constexpr int LPR = RowGeo<HD>::LPR;
-    const int g = (blockIdx.x * blockDim.x + threadIdx.x) / LPR, sub = threadIdx.x % LPR;
-    if (g >= a.B * a.H) return;
-    const float* w = a.ws + (size_t)g * a.splits * kPartStride<HD>;
-    float mx = kNegInf;
-    for (int s = 0; s < a.splits; ++s) mx = fmaxf(mx, w[s * kPartStride<HD> + HD]);
-    float o[8] = {0, 0, 0, 0, 0, 0, 0, 0};
-    float tot = 0.f;
-    if (mx != kNegInf) {
-        for (int s = 0; s < a.splits; ++s) {
-            const float* ws = w + s * kPartStride<HD>;
-            float c = ex2(ws[HD] - mx);
-            tot += c;
-            float4 x = *reinterpret_cast<const float4*>(ws + sub * 8);
-            float4 y = *reinterpret_cast<const float4*>(ws + sub * 8 + 4);
-            o[0] = fmaf(c, x.x, o[0]); o[1] = fmaf(c, x.y, o[1]); o[2] = fmaf(c, x.z, o[2]); o[3] = fmaf(c, x.w, o[3]);
-            o[4] = fmaf(c, y.x, o[4]); o[5] = fmaf(c, y.y, o[5]); o[6] = fmaf(c, y.z, o[6]); o[7] = fmaf(c, y.w, o[7]);
-        }
-        float inv = 1.f / tot;
-#pragma unroll
-        for (int i = 0; i < 8; ++i) o[i] *= inv;
-    }
-    *reinterpret_cast<uint4*>(reinterpret_cast<bf16*>(a.out) + (size_t)g * HD + sub * 8) = pack8(o);
-}
-
-template <int HD>
-static cudaError_t launch_decode_t(const DecodeArgs& a, cudaStream_t stream)
-{
-    const int bh = a.B * a.H;
-    cudaError_t e = launch_block_decode_ring(a, stream);
-    if (e != cudaSuccess || a.splits == 1) return e;
-    constexpr int LPR = RowGeo<HD>::LPR;
-    const int groups_per_cta = 128 / LPR;
-    decode_merge_kernel<HD><<<(bh + groups_per_cta - 1) / groups_per_cta, 128, 0, stream>>>(a);
-    return cudaGetLastError();
-}
-
-cudaError_t launch_block_decode(const DecodeArgs& a, cudaStream_t stream)
-{
-    return a.hd == 64 ? launch_decode_t<64>(a, stream) : launch_decode_t<128>(a, stream);
 }
 
 // ---------------------------------------------------------------------------------------

@@ -49,10 +49,14 @@ extern "C" bt_status bt_block_decode_attn_noalloc(const bt_config* cfg, const bt
     const size_t need = bt_workspace_bytes(cfg);
     if (need > (size_t)BT_STATIC_WORKSPACE_BYTES) return BT_ERR_WORKSPACE;
     void* ws = nullptr;
-    if (need) {
+    if (need && bt_decode_splits(cfg) > 1) {
         bt_status st = static_ws_on_current_device(&ws);
         if (st != BT_OK) return st;
+        // configs of different shapes share the array, and one config's partial results may lie where
+        // another's arrival counters do: the counters are zeroed (a memset node, no allocation) every time
+        st = bt_workspace_init(cfg, ws, (size_t)BT_STATIC_WORKSPACE_BYTES, stream);
+        if (st != BT_OK) return st;
     }
-    return bt_block_decode_attn(cfg, cache, layer, q, out, ws, need ? (size_t)BT_STATIC_WORKSPACE_BYTES : 0,
+    return bt_block_decode_attn(cfg, cache, layer, q, out, ws, ws ? (size_t)BT_STATIC_WORKSPACE_BYTES : 0,
                                 dev_status, stream);
 }

@@ -11,14 +11,15 @@ from . import binding as bt
 
 class BlockDecodeStep:
     """One block-decoder decode step over all layers (section 2.3): per layer, append the new
-    block's K,V row, then attend causally over the whole block cache.
+    block's K,V row, then attend causally over the whole block cache - one fused launch per
+    layer (bt_block_decode_step), or with ``fused=False`` the two separate calls.
 
     The caches are pre-filled to ``ctx_blocks - 1`` rows so that after the append every sequence
     attends over ``ctx_blocks`` rows.  ``rewind()`` puts the lengths back so a step can be repeated.
     """
 
-    def __init__(self, w, device="cuda", fill=None):
-        self.w, self.device = w, device
+    def __init__(self, w, device="cuda", fill=None, fused=True):
+        self.w, self.device, self.fused = w, device, fused
         self.cfg = bt.make_config(w.batch, w.heads, w.head_dim, w.block_len, w.prefix_len, w.max_blocks, w.n_layers)
         shape = (w.n_layers, w.batch, w.heads, w.max_blocks, w.head_dim)
         if fill is None:
@@ -35,8 +36,8 @@ class BlockDecodeStep:
         self.out = torch.empty(io, dtype=torch.bfloat16, device=device)
         self.ws = bt.alloc_workspace(self.cfg, device)
         self.status = torch.zeros(1, dtype=torch.int32, device=device)
-        # append + attention per layer, plus the merge pass when the row range is split
-        self.launches_per_step = w.n_layers * (2 + (1 if bt.bt_decode_splits(self.cfg) > 1 else 0))
+        # per layer one fused launch, or append + attention (split row ranges are merged inside the launch)
+        self.launches_per_step = w.n_layers * (1 if fused else 2)
         self._host = None
 
     def rewind(self):
@@ -46,26 +47,36 @@ class BlockDecodeStep:
         """Enqueue one step.  attn_events: optional list receiving (start, stop) CUDA events around
         each attention launch."""
         for l in range(self.w.n_layers):
-            bt.bt_block_kv_append(self.cfg, self.cache, l, self.k_new[l], self.v_new[l], n_new=1, dev_status=self.status)
+            if not self.fused:
+                bt.bt_block_kv_append(self.cfg, self.cache, l, self.k_new[l], self.v_new[l], n_new=1, dev_status=self.status)
             if attn_events is not None:
                 e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
                 e0.record()
-            bt.bt_block_decode_attn(self.cfg, self.cache, l, self.q[l], self.out[l], self.ws, dev_status=self.status)
+            self._layer(l)
             if attn_events is not None:
                 e1.record()
                 attn_events.append((e0, e1))
+
+    def _layer(self, l):
+        """The attention launch of layer l: with the append fused in, or after a separate append."""
+        if self.fused:
+            bt.bt_block_decode_step(self.cfg, self.cache, l, self.q[l], self.k_new[l], self.v_new[l], self.out[l], self.ws,
+                                    dev_status=self.status)
+        else:
+            bt.bt_block_decode_attn(self.cfg, self.cache, l, self.q[l], self.out[l], self.ws, dev_status=self.status)
 
     def _capture(self, events):
         g = torch.cuda.CUDAGraph()
         with torch.cuda.graph(g):
             self.rewind()
             for l in range(self.w.n_layers):
-                bt.bt_block_kv_append(self.cfg, self.cache, l, self.k_new[l], self.v_new[l], n_new=1, dev_status=self.status)
+                if not self.fused:
+                    bt.bt_block_kv_append(self.cfg, self.cache, l, self.k_new[l], self.v_new[l], n_new=1, dev_status=self.status)
                 if events is not None:
                     e0 = torch.cuda.Event(enable_timing=True, external=True)
                     e1 = torch.cuda.Event(enable_timing=True, external=True)
                     e0.record()
-                bt.bt_block_decode_attn(self.cfg, self.cache, l, self.q[l], self.out[l], self.ws, dev_status=self.status)
+                self._layer(l)
                 if events is not None:
                     e1.record()
                     events.append((e0, e1))
@@ -269,7 +280,7 @@ class GenerationRun:
         self.n_gen_blocks = w.gen_tokens // w.block_len
         self.graph = None
         self.launches_prefill = 2 * L
-        self.launches_per_block = L * (w.block_len + 2 + (1 if bt.bt_decode_splits(self.cfg) > 1 else 0))
+        self.launches_per_block = L * (w.block_len + 1)   # L_B token steps + one fused block step, per layer
 
     def start(self):
         """Empty caches, then the prompt: prefill attention and bulk append per layer."""
@@ -289,8 +300,8 @@ class GenerationRun:
                 bt.bt_token_decode_attn(self.cfg, self.local, l, self.tq[r, j, l], self.tk[r, j, l], self.tv[r, j, l], self.tout[l],
                                         n_q=1, reset_first=(j == 0), dev_status=self.status)
         for l in range(w.n_layers):
-            bt.bt_block_kv_append(self.cfg, self.block, l, self.bk[r, l], self.bv[r, l], n_new=1, dev_status=self.status)
-            bt.bt_block_decode_attn(self.cfg, self.block, l, self.bq[r, l], self.bout[l], self.ws, dev_status=self.status)
+            bt.bt_block_decode_step(self.cfg, self.block, l, self.bq[r, l], self.bk[r, l], self.bv[r, l], self.bout[l], self.ws,
+                                    dev_status=self.status)
 
     def capture(self):
         """One pass over the input ring (ring generated blocks) as a CUDA graph."""

@@ -36,10 +36,11 @@ def test_version_and_status_strings(bt):
 
 def test_split_choice_and_workspace(bt):
     big = bt.make_config(256, 16, 64, 4, 1, 512, 12)
-    assert bt.bt_decode_splits(big) == 1 and bt.bt_workspace_bytes(big) == 0
+    counters = lambda B, H: (B * H + B) * 4   # arrival counters: one per (b,h), one per sequence
+    assert bt.bt_decode_splits(big) == 1 and bt.bt_workspace_bytes(big) == counters(256, 16)
     tiny = bt.make_config(4, 8, 64, 4, 1, 64, 2)
     s = bt.bt_decode_splits(tiny)
-    assert s > 1 and bt.bt_workspace_bytes(tiny) == s * 4 * 8 * 68 * 4
+    assert s > 1 and bt.bt_workspace_bytes(tiny) == s * 4 * 8 * 68 * 4 + counters(4, 8)
     forced = bt.make_config(4, 8, 64, 4, 1, 64, 2, decode_splits=7)
     assert bt.bt_decode_splits(forced) == 7
     bad = bt.make_config(4, 8, 48, 4, 1, 64, 2)
@@ -72,6 +73,11 @@ def test_host_detectable_errors_return_before_launch(bt):
     # workspace too small when the row range is split
     assert L.bt_block_decode_attn(ref(cfg), ref(bc), 0, fake, fake, None, 0, None, None) == bt.BT_ERR_WORKSPACE
     assert L.bt_block_decode_attn(ref(cfg), ref(bc), 0, fake, fake, fake, 16, None, None) == bt.BT_ERR_WORKSPACE
+    # the fused step needs one always; the initialiser checks its size too
+    assert L.bt_block_decode_step(ref(cfg), ref(bc), 0, fake, fake, fake, fake, None, 0, None, None) == bt.BT_ERR_WORKSPACE
+    assert L.bt_block_decode_step(ref(cfg), ref(bc), 0, fake, None, fake, fake, fake, 1 << 20, None, None) == bt.BT_ERR_NULL
+    assert L.bt_workspace_init(ref(cfg), fake, 16, None) == bt.BT_ERR_WORKSPACE
+    assert L.bt_workspace_init(ref(cfg), None, 1 << 20, None) == bt.BT_ERR_NULL
     assert L.bt_block_decode_attn(ref(cfg), ref(bc), 0, None, fake, fake, 1 << 20, None, None) == bt.BT_ERR_NULL
     # local cache
     assert L.bt_local_kv_reset(ref(cfg), None, 0, None, None) == bt.BT_ERR_NULL

@@ -41,12 +41,13 @@ class Guarded:
 def test_block_path_touches_nothing_outside_its_rows(bt):
     rng = np.random.default_rng(7)
     B, H, hd, N = 37, 5, 64, 96
-    for trial, splits in enumerate((0, 1, 3)):
+    for trial, (splits, fused) in enumerate(((0, False), (1, False), (3, False), (0, True), (1, True), (3, True))):
         cfg = bt.make_config(B, H, hd, 4, 1, N, 1, decode_splits=splits)
         k, v = Guarded((1, B, H, N, hd), torch.bfloat16), Guarded((1, B, H, N, hd), torch.bfloat16)
         ln = Guarded((1, B), torch.int32)
         q, kn, vn, out = (Guarded((B, H, 1, hd), torch.bfloat16) for _ in range(4))
         ws = Guarded((max(bt.bt_workspace_bytes(cfg), 4) // 4,), torch.float32)
+        bt.bt_workspace_init(cfg, ws.t)  # zeroes the arrival counters; the partial results keep the pattern
         lens = rng.integers(0, N + 1, B).astype(np.int32)
         lens[0], lens[1] = 0, N  # an empty cache (append fits) and a full one (append must be refused)
         kb, vb = gen.normal_bf16_bits(300 + trial, 1, (B, H, N, hd)), gen.normal_bf16_bits(300 + trial, 2, (B, H, N, hd))
@@ -55,8 +56,11 @@ def test_block_path_touches_nothing_outside_its_rows(bt):
         q.t.copy_(to_dev(qb)); kn.t.copy_(to_dev(knb)); vn.t.copy_(to_dev(vnb))
         cache = bt.BlockCache(cfg, k=k.t, v=v.t, length=ln.t)
         st = status_word()
-        bt.bt_block_kv_append(cfg, cache, 0, kn.t, vn.t, n_new=1, dev_status=st)
-        bt.bt_block_decode_attn(cfg, cache, 0, q.t[:, :, 0], out.t[:, :, 0], ws.t, dev_status=st)
+        if fused:
+            bt.bt_block_decode_step(cfg, cache, 0, q.t[:, :, 0], kn.t, vn.t, out.t[:, :, 0], ws.t, dev_status=st)
+        else:
+            bt.bt_block_kv_append(cfg, cache, 0, kn.t, vn.t, n_new=1, dev_status=st)
+            bt.bt_block_decode_attn(cfg, cache, 0, q.t[:, :, 0], out.t[:, :, 0], ws.t, dev_status=st)
         torch.cuda.synchronize()
         oc = oracle.Cache(B, H, N, hd)
         oc.k[...], oc.v[...], oc.len[...] = kb, vb, lens
@@ -68,7 +72,7 @@ def test_block_path_touches_nothing_outside_its_rows(bt):
         assert np.array_equal(gen.torch_to_bits(k.t[0]), oc.k) and np.array_equal(gen.torch_to_bits(v.t[0]), oc.v)
         assert np.array_equal(ln.t[0].cpu().numpy(), oc.len) and oc.len[1] == N and oc.len[0] == 1
         assert np.array_equal(gen.torch_to_bits(q.t), qb) and np.array_equal(gen.torch_to_bits(kn.t), knb)
-        assert_close(out.t[:, :, 0], ref, f"guarded decode, splits {splits}")
+        assert_close(out.t[:, :, 0], ref, f"guarded decode, splits {splits}, fused {fused}")
         assert st.item() == bt.BT_DEV_OVERFLOW == int(oc.status[0])
 
 

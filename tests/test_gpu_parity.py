@@ -177,7 +177,8 @@ def test_block_decode_ragged_lengths_poison_and_splits(bt, hd, splits):
     cache = bt.BlockCache(cfg)
     fill_block_cache(bt, cfg, cache, 0, kp, vp, lens)
     ws = bt.alloc_workspace(cfg)
-    ws.fill_(float("nan"))  # the workspace needs no initialisation
+    ws.fill_(float("nan"))  # the partial results need no initialisation, only the arrival counters do
+    bt.bt_workspace_init(cfg, ws)
     st = status_word()
     out = torch.full((B, H, hd), 7.0, dtype=torch.bfloat16, device="cuda")
     bt.bt_block_decode_attn(cfg, cache, 0, to_dev(q), out, ws, dev_status=st)
