@@ -198,6 +198,11 @@ def workload_config(w, name):
         c.update(workload="block_decode: BASELINE configs[1], per layer append 1 block row then attend over 512 rows",
                  ctx_blocks=w.ctx_blocks, context_tokens=w.ctx_blocks * w.block_len,
                  l2="no flush: 6.4 GB of KV per step, 537 MB per launch, L2 is 126 MB")
+    elif name == "block_decode_16k":
+        c.update(workload="block_decode_16k: the block-decoder decode step at a 16K-token context (4096 block rows), batch 64 "
+                          "(with --batch 1..16: the small-batch case, row ranges split across the GPU)",
+                 ctx_blocks=w.ctx_blocks, context_tokens=w.ctx_blocks * w.block_len,
+                 l2="no flush: 1.07 GB of KV per launch at batch 64; at batch 1 a launch's 16.8 MB fit L2 but the 12 layers' 201 MB do not")
     elif name == "token_decode":
         c.update(workload="token_decode: BASELINE configs[2], fused reset+append+local attention, 12 launches per token step",
                  l2="no flush: inputs rotate over a ring larger than L2")
@@ -265,10 +270,11 @@ def run_gpu(args):
 
     sampler = ClockSampler(local_rank)
     kern_events = []
-    if args.workload == "block_decode":
+    if args.workload in ("block_decode", "block_decode_16k"):
         run = harness.BlockDecodeStep(w, fill=fill)
         tokens_per_step = w.batch * w.block_len
-        # a bench step = one CUDA-graph replay of (put the lengths back, then 12 x (append + attention)).
+        # a bench step = one CUDA-graph replay of (put the lengths back, then 12 launches, each appending the
+        # layer's new row and attending over the cache including it).
         # The per-launch time of the attention kernel comes from a twin graph of the same step with timing
         # events around every attention launch, replayed right after the timed region (events inside the
         # timed graph would lengthen the step they measure).
@@ -346,7 +352,7 @@ def run_gpu(args):
 
     torch.cuda.synchronize()
     kern_ms_events = statistics.mean(a.elapsed_time(b) for a, b in kern_events) if kern_events else None
-    if args.workload == "block_decode":
+    if args.workload in ("block_decode", "block_decode_16k"):
         kern_ms = ms_attn
     elif kern_events:
         kern_ms = kern_ms_events
@@ -400,7 +406,7 @@ def main():
     ap.add_argument("--steps", type=int, default=0, help="timed steps (default 200; 3 for the sweep, whose step is a whole generation)")
     ap.add_argument("--warmup", type=int, default=3)
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
-    ap.add_argument("--workload", default="block_decode", choices=["block_decode", "token_decode", "block_prefill", "block_prefill_8k", "sweep"])
+    ap.add_argument("--workload", default="block_decode", choices=["block_decode", "block_decode_16k", "token_decode", "block_prefill", "block_prefill_8k", "sweep"])
     ap.add_argument("--block-len", type=int, default=4, help="L_B of the generation sweep (1, 2, 4 or 8)")
     ap.add_argument("--prefix-len", type=int, default=0, help="token_decode: prefix length P (default 1 = BASELINE configs[2]; 2 = the paper's main setting)")
     ap.add_argument("--no-cpu-baseline", action="store_true")

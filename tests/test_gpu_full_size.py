@@ -52,6 +52,32 @@ def test_block_decode_step_full_size(bt):
         assert_close(run.out[l][seqs][:, :, 0], ref, f"full-size block decode layer {l}")
 
 
+@pytest.mark.parametrize("batch", [64, 1])
+def test_block_decode_step_long_context(bt, batch):
+    """The 16K-token context (4096 block rows): the bench batch, unsplit, and a single sequence, whose
+    row ranges are split across the GPU and merged inside the launch."""
+    from paper_2406_02657_b200 import harness
+    w = configs.scaled(configs.BLOCK_DECODE_16K, batch=batch, n_layers=2)
+    run = harness.BlockDecodeStep(w, fill=_fill(w))
+    assert (bt.bt_decode_splits(run.cfg) > 1) == (batch == 1)
+    for _ in range(2):   # twice on the same workspace
+        run.rewind()
+        run.out.zero_()
+        run.step()
+        torch.cuda.synchronize()
+        assert run.status.item() == 0 and (run.cache.len == w.ctx_blocks).all()
+        assert torch.equal(run.cache.k[:, :, :, w.ctx_blocks - 1], run.k_new[:, :, :, 0])
+        assert torch.equal(run.cache.v[:, :, :, w.ctx_blocks - 1], run.v_new[:, :, :, 0])
+        seqs = sorted({0, batch // 2, batch - 1})
+        for l in range(w.n_layers):
+            c = oracle.Cache(len(seqs), w.heads, w.max_blocks, w.head_dim)
+            c.k[...] = gen.torch_to_bits(run.cache.k[l][seqs])
+            c.v[...] = gen.torch_to_bits(run.cache.v[l][seqs])
+            c.len[...] = w.ctx_blocks
+            ref = oracle.block_decode_attn(c, gen.torch_to_bits(run.q[l][seqs][:, :, 0]))
+            assert_close(run.out[l][seqs][:, :, 0], ref, f"16K-context block decode, batch {batch}, layer {l}")
+
+
 def test_block_decode_step_through_host_buffers(bt):
     """The e2e path of bench.py: the same step driven from pinned host buffers through
     bt_block_decode_step_host (per-layer calls on several streams) gives the device-resident step's

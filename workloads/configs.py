@@ -39,6 +39,11 @@ TINY = Workload("tiny", batch=4, heads=8, head_dim=64, block_len=4, prefix_len=1
 BLOCK_DECODE = Workload("block_decode", batch=256, heads=16, head_dim=64, block_len=4, prefix_len=1,
                         n_layers=12, max_blocks=512, ctx_blocks=512, seed=1002)
 
+# config 2b: the same step at a context eight times longer (16K tokens -> 4096 block entries; the paper's
+# long-context comparison raises the context four- and eightfold), batch sized to a 13 GB cache
+BLOCK_DECODE_16K = Workload("block_decode_16k", batch=64, heads=16, head_dim=64, block_len=4, prefix_len=1,
+                            n_layers=12, max_blocks=4096, ctx_blocks=4096, seed=1012)
+
 # config 3: token-decoder local decode, 4096 sequences, local cache 1 prefix + up to L_B tokens
 TOKEN_DECODE = Workload("token_decode", batch=4096, heads=16, head_dim=64, block_len=4, prefix_len=1,
                         n_layers=12, max_blocks=1, gen_tokens=4096, seed=1003)
@@ -66,4 +71,4 @@ def scaled(w: Workload, **kw) -> Workload:
     return replace(w, **kw)
 
 
-BY_NAME = {w.name: w for w in (TINY, BLOCK_DECODE, TOKEN_DECODE, BLOCK_PREFILL, BLOCK_PREFILL_8K)}
+BY_NAME = {w.name: w for w in (TINY, BLOCK_DECODE, BLOCK_DECODE_16K, TOKEN_DECODE, BLOCK_PREFILL, BLOCK_PREFILL_8K)}
