@@ -148,6 +148,25 @@ bt_status bt_block_decode_step(const bt_config* cfg, bt_block_cache* cache, int 
                                size_t workspace_bytes, uint32_t* dev_status, void* stream);
 
 /*
+ * Decode step of the "densified" block decoder the paper proposes as future work (appendix
+ * "Discussion and future works": a block is represented by L_B sub-block tokens instead of one, so
+ * a step appends L_B rows and runs L_B queries while the cache is fetched once).  For each
+ * sequence b with len[b] + n_q <= N_max: rows len[b] .. len[b]+n_q-1 of every head receive
+ * k_new / v_new [B][H][n_q][hd]; query i of q [B][H][n_q][hd] attends to rows 0 .. len[b]+i
+ * (every cached row and the new rows 0..i); out [B][H][n_q][hd]; len[b] += n_q.  A sequence
+ * without room for all n_q rows is left as it is, every query attends over its len[b] rows, and
+ * BT_DEV_OVERFLOW is raised.  n_q = 1 computes what bt_block_decode_step computes.
+ * Scores and weighted sums run on the tensor cores (bf16 inputs, fp32 accumulation; the softmax
+ * weights are rounded to bf16 where they meet V).  Supported: head_dim 64, 1 <= n_q <= 8,
+ * N_max >= 32, all pointers 16-byte aligned; otherwise BT_ERR_UNSUPPORTED.  The row range is
+ * never split.  workspace: required, as for bt_block_decode_step.
+ */
+bt_status bt_block_decode_step_multi(const bt_config* cfg, bt_block_cache* cache, int layer, const void* q,
+                                     const void* k_new, const void* v_new, int n_q, void* out,
+                                     void* workspace, size_t workspace_bytes, uint32_t* dev_status,
+                                     void* stream);
+
+/*
  * bt_block_decode_attn for callers that cannot supply a workspace.  (The paper has no
  * counterpart: this is a property of the library, not of the method.)  It computes exactly what
  * bt_block_decode_attn computes, with the per-split partials kept in a fixed array inside the

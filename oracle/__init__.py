@@ -154,6 +154,29 @@ def token_decode_attn(c: Cache, q, k_new, v_new, reset_first=False, reset_mask=N
     return out
 
 
+def block_decode_step_multi(c: Cache, q, k_new, v_new, scale=None, f32=False):
+    """Decode step of the densified block decoder (appendix "Discussion and future works"): a block
+    is L_B sub-block tokens, so a step appends m rows and runs m queries, query i seeing every cached
+    row and the new rows 0..i.  q, k_new, v_new [B,H,m,hd] -> out [B,H,m,hd].
+
+    Written as the definition: the m rows are appended (all of them or, for a sequence without room,
+    none, as kv_append does), then query i is a plain decode over the first len_before + i + 1 rows.
+    A sequence that had no room keeps its rows and every query attends over them."""
+    q = _u16(q)
+    m = q.shape[2]
+    assert q.shape == (c.B, c.H, m, c.hd)
+    before = c.len.copy()
+    kv_append(c, k_new, v_new)
+    after = c.len.copy()
+    dt, _ = _real(f32)
+    out = np.zeros((c.B, c.H, m, c.hd), dt)
+    for i in range(m):
+        c.len[...] = np.where(after > before, before + i + 1, before)
+        out[:, :, i] = block_decode_attn(c, np.ascontiguousarray(q[:, :, i]), scale=scale, f32=f32)
+    c.len[...] = after
+    return out
+
+
 def block_prefill_attn(q, k, v, scale=None, f32=False, kv_seq_stride=None):
     """Dense causal attention over T blocks; q [B,H,T,hd]; k,v [B,H,stride,hd] -> out [B,H,T,hd]."""
     q, k, v = _u16(q), _u16(k), _u16(v)

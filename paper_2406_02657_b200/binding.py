@@ -21,7 +21,7 @@ EXPORTS = [
     "bt_version", "bt_status_string", "bt_decode_splits", "bt_workspace_bytes", "bt_block_kv_append",
     "bt_block_decode_attn", "bt_local_kv_reset", "bt_local_kv_append", "bt_token_decode_attn",
     "bt_block_prefill_attn", "bt_block_decode_step_host", "bt_block_decode_attn_noalloc",
-    "bt_workspace_init", "bt_block_decode_step",
+    "bt_workspace_init", "bt_block_decode_step", "bt_block_decode_step_multi",
 ]
 
 
@@ -64,6 +64,7 @@ def _load() -> ctypes.CDLL:
     lib.bt_block_decode_attn.argtypes = [cfgp, ctypes.POINTER(bt_block_cache), i32, vp, vp, vp, u64, vp, vp]
     lib.bt_workspace_init.argtypes = [cfgp, vp, u64, vp]
     lib.bt_block_decode_step.argtypes = [cfgp, ctypes.POINTER(bt_block_cache), i32, vp, vp, vp, vp, vp, u64, vp, vp]
+    lib.bt_block_decode_step_multi.argtypes = [cfgp, ctypes.POINTER(bt_block_cache), i32, vp, vp, vp, i32, vp, vp, u64, vp, vp]
     lib.bt_local_kv_reset.argtypes = [cfgp, ctypes.POINTER(bt_local_cache), i32, vp, vp]
     lib.bt_local_kv_append.argtypes = [cfgp, ctypes.POINTER(bt_local_cache), i32, vp, vp, i32, vp, vp]
     lib.bt_token_decode_attn.argtypes = [cfgp, ctypes.POINTER(bt_local_cache), i32, vp, vp, vp, i32, i32, vp, vp, vp, vp]
@@ -178,6 +179,15 @@ def bt_block_decode_step(cfg, cache: BlockCache, layer, q, k_new, v_new, out, wo
     _check(_lib.bt_block_decode_step(ctypes.byref(cfg), ctypes.byref(cache.c), layer, _ptr(q), _ptr(k_new), _ptr(v_new),
                                      _ptr(out), _ptr(workspace), workspace.numel() * workspace.element_size(),
                                      _ptr(dev_status), _stream(stream)), "bt_block_decode_step")
+
+
+def bt_block_decode_step_multi(cfg, cache: BlockCache, layer, q, k_new, v_new, out, workspace, n_q=None, dev_status=None,
+                               stream=None):
+    """Append n_q rows and run n_q queries (query i sees the cache and new rows 0..i), one launch."""
+    n_q = q.shape[2] if n_q is None else n_q
+    _check(_lib.bt_block_decode_step_multi(ctypes.byref(cfg), ctypes.byref(cache.c), layer, _ptr(q), _ptr(k_new), _ptr(v_new),
+                                           n_q, _ptr(out), _ptr(workspace), workspace.numel() * workspace.element_size(),
+                                           _ptr(dev_status), _stream(stream)), "bt_block_decode_step_multi")
 
 
 BT_STATIC_WORKSPACE_BYTES = 2 << 20

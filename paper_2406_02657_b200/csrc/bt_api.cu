@@ -192,6 +192,37 @@ bt_status bt_block_decode_step(const bt_config* cfg, bt_block_cache* cache, int 
     return decode_launch(cfg, cache, layer, q, k_new, v_new, out, workspace, workspace_bytes, dev_status, stream);
 }
 
+bt_status bt_block_decode_step_multi(const bt_config* cfg, bt_block_cache* cache, int layer, const void* q,
+                                     const void* k_new, const void* v_new, int n_q, void* out, void* workspace,
+                                     size_t workspace_bytes, uint32_t* dev_status, void* stream)
+{
+    bt_status st = check_config(cfg, layer);
+    if (st != BT_OK) return st;
+    if (!cache || !cache->k || !cache->v || !cache->len || !q || !k_new || !v_new || !out) return BT_ERR_NULL;
+    if (n_q <= 0) return BT_ERR_SHAPE;
+    if (n_q > cfg->max_blocks) return BT_ERR_CAPACITY;
+    if (!workspace || workspace_bytes < bt_workspace_bytes(cfg)) return BT_ERR_WORKSPACE;
+    bt::CacheView v = block_view(cfg, cache, layer);
+    bt::MultiDecodeArgs a;
+    a.q = q;
+    a.k_new = k_new;
+    a.v_new = v_new;
+    a.k = v.k;
+    a.v = v.v;
+    a.len = v.len;
+    a.out = out;
+    a.counters = (int32_t*)((char*)workspace + partial_bytes(cfg));
+    a.dev_status = dev_status;
+    a.B = cfg->batch;
+    a.H = cfg->heads;
+    a.hd = cfg->head_dim;
+    a.n_max = cfg->max_blocks;
+    a.m = n_q;
+    a.scale_log2 = scale_log2(cfg);
+    if (!bt::multi_decode_supported(a)) return BT_ERR_UNSUPPORTED;
+    return cuda_status(bt::launch_block_decode_multi(a, (cudaStream_t)stream));
+}
+
 bt_status bt_local_kv_reset(const bt_config* cfg, bt_local_cache* cache, int layer, const uint8_t* seq_mask,
                             void* stream)
 {

@@ -42,6 +42,23 @@ struct DecodeArgs {
 // The streaming kernel: per-item results, or per-split partials merged by the split that finishes last.
 cudaError_t launch_block_decode(const DecodeArgs& a, cudaStream_t stream);
 
+// Decode step with m queries and m new rows per (sequence, head) (query i sees the cache and new rows 0..i).
+struct MultiDecodeArgs {
+    const void* q;       // [B][H][m][hd]
+    const void* k_new;   // [B][H][m][hd]
+    const void* v_new;
+    void* k;             // layer base, [B][H][N_max][hd]
+    void* v;
+    int32_t* len;        // [B]
+    void* out;           // [B][H][m][hd]
+    int32_t* counters;   // decode workspace counters: [B*H] (unused here) then [B], zero on entry and on exit
+    uint32_t* dev_status;
+    int B, H, hd, n_max, m;
+    float scale_log2;
+};
+bool multi_decode_supported(const MultiDecodeArgs& a);
+cudaError_t launch_block_decode_multi(const MultiDecodeArgs& a, cudaStream_t stream);
+
 struct TokenArgs {
     void* kv;            // layer base, [B][H][C][2][hd]
     int32_t* len;        // [B]

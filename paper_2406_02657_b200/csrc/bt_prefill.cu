@@ -24,6 +24,7 @@
 
 #include "bt_common.cuh"
 #include "bt_kernels.h"
+#include "bt_tensor_map.h"
 
 namespace bt {
 namespace pf {
@@ -770,39 +771,12 @@ block_prefill_tc_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_c
     }
 }
 
-// ---- host side: tensor maps through the driver entry point (no link-time dependency on libcuda)
-using EncodeFn = CUresult (*)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*, const cuuint64_t*,
-                              const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave, CUtensorMapSwizzle,
-                              CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
-
-static EncodeFn encode_fn()
-{
-    static EncodeFn fn = nullptr;
-    static bool tried = false;
-    if (!tried) {
-        tried = true;
-        void* f = nullptr;
-        cudaDriverEntryPointQueryResult q;
-        if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &f, cudaEnableDefault, &q) == cudaSuccess &&
-            q == cudaDriverEntryPointSuccess)
-            fn = reinterpret_cast<EncodeFn>(f);
-    }
-    return fn;
-}
-
+// ---- host side
 // [slabs][rows][hd] bf16 with `stride_rows` rows between slabs; box = 64 x 128 x 1, 128-byte swizzle,
 // rows past `rows` read as zeros.
 static bool make_map(CUtensorMap* m, const void* ptr, int hd, int rows, long long stride_rows, long long slabs)
 {
-    EncodeFn fn = encode_fn();
-    if (!fn) return false;
-    cuuint64_t dims[3] = {(cuuint64_t)hd, (cuuint64_t)rows, (cuuint64_t)slabs};
-    cuuint64_t strides[2] = {(cuuint64_t)hd * 2, (cuuint64_t)stride_rows * hd * 2};
-    cuuint32_t box[3] = {64, 128, 1};
-    cuuint32_t estr[3] = {1, 1, 1};
-    return fn(m, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 3, const_cast<void*>(ptr), dims, strides, box, estr,
-              CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
-              CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
+    return make_slab_map(m, ptr, hd, rows, stride_rows, slabs, 128);
 }
 
 static int gcd_int(int a, int b)
@@ -859,7 +833,7 @@ static cudaError_t launch_t(const PrefillArgs& a, uint32_t* dev_status, cudaStre
 bool prefill_tc_supported(const PrefillArgs& a)
 {
     auto al = [](const void* p) { return (reinterpret_cast<uintptr_t>(p) & 15u) == 0; };
-    return (a.hd == 64 || a.hd == 128) && al(a.q) && al(a.k) && al(a.v) && al(a.out) && pf::encode_fn() != nullptr;
+    return (a.hd == 64 || a.hd == 128) && al(a.q) && al(a.k) && al(a.v) && al(a.out) && tensor_map_encode_fn() != nullptr;
 }
 
 cudaError_t launch_block_prefill_tc(const PrefillArgs& a, uint32_t* dev_status, cudaStream_t stream)

@@ -200,6 +200,45 @@ def test_cached_decode_equals_full_recompute():
     assert np.array_equal(c.k, k) and np.array_equal(c.v, v) and c.status[0] == 0
 
 
+def test_densified_step_is_the_matching_rows_of_dense_causal_attention():
+    """The densified block decoder's step (m sub-block rows and queries at once) changes the schedule,
+    not the function: steps of m rows reproduce the rows of the dense causal prefill over all
+    sub-block tokens; and m = 1 is the ordinary append + decode."""
+    B, H, hd, m, steps = 2, 3, 16, 4, 5
+    T = m * steps
+    q, k, v = rnd(15, 0, (B, H, T, hd)), rnd(15, 1, (B, H, T, hd)), rnd(15, 2, (B, H, T, hd))
+    full = oracle.block_prefill_attn(q, k, v)
+    c = oracle.Cache(B, H, T, hd)
+    for s_ in range(steps):
+        sl = slice(s_ * m, (s_ + 1) * m)
+        out = oracle.block_decode_step_multi(c, q[:, :, sl], k[:, :, sl], v[:, :, sl])
+        assert (c.len == (s_ + 1) * m).all()
+        assert np.array_equal(out, full[:, :, sl])
+    assert np.array_equal(c.k, k) and np.array_equal(c.v, v) and c.status[0] == 0
+    # m = 1: append then decode
+    c1, c2 = oracle.Cache(B, H, 8, hd), oracle.Cache(B, H, 8, hd)
+    for t in range(3):
+        a_ = oracle.block_decode_step_multi(c1, q[:, :, t:t + 1], k[:, :, t:t + 1], v[:, :, t:t + 1])
+        oracle.kv_append(c2, k[:, :, t:t + 1], v[:, :, t:t + 1])
+        assert np.array_equal(a_[:, :, 0], oracle.block_decode_attn(c2, np.ascontiguousarray(q[:, :, t])))
+
+
+def test_densified_step_without_room_appends_nothing():
+    """All m rows or none: a sequence one row short of room is left as it is, flagged, and every query
+    sees exactly its old rows (so the m outputs of one head differ only through their queries)."""
+    B, H, hd, N, m = 2, 1, 16, 6, 4
+    c = oracle.Cache(B, H, N, hd)
+    c.k[...], c.v[...] = rnd(16, 1, (B, H, N, hd)), rnd(16, 2, (B, H, N, hd))
+    c.len[...] = [2, 3]
+    k0 = c.k.copy()
+    q = np.repeat(rnd(16, 0, (B, H, 1, hd)), m, axis=2)   # the same query m times
+    out = oracle.block_decode_step_multi(c, q, rnd(16, 3, (B, H, m, hd)), rnd(16, 4, (B, H, m, hd)))
+    assert c.len.tolist() == [6, 3] and c.status[0] == 1          # BT_DEV_OVERFLOW
+    assert np.array_equal(c.k[1], k0[1]) and not np.array_equal(c.k[0], k0[0])
+    assert all(np.array_equal(out[1, :, i], out[1, :, 0]) for i in range(m))       # same rows, same query
+    assert not np.array_equal(out[0, :, 1], out[0, :, 0])                            # causal: one more row each
+
+
 def test_block_length_one_is_vanilla_causal_attention():
     """At L_B = 1 every token is its own block, so block-decoder attention over the block cache
     is token-level causal attention (the library routine, float64)."""
