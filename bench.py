@@ -203,6 +203,11 @@ def workload_config(w, name):
                           "(with --batch 1..16: the small-batch case, row ranges split across the GPU)",
                  ctx_blocks=w.ctx_blocks, context_tokens=w.ctx_blocks * w.block_len,
                  l2="no flush: 1.07 GB of KV per launch at batch 64; at batch 1 a launch's 16.8 MB fit L2 but the 12 layers' 201 MB do not")
+    elif name == "dense_decode":
+        c.update(workload="dense_decode: the densified block decoder of the paper's future-work discussion - one cache row per "
+                          "token (2048 rows), a step appends L_B = 4 rows and runs 4 queries per (sequence, head), 12 layers",
+                 ctx_rows=w.ctx_blocks, context_tokens=w.ctx_blocks,
+                 l2="no flush: 2.1 GB of KV per launch")
     elif name == "token_decode":
         c.update(workload="token_decode: BASELINE configs[2], fused reset+append+local attention, 12 launches per token step",
                  l2="no flush: inputs rotate over a ring larger than L2")
@@ -298,6 +303,21 @@ def run_gpu(args):
         dom = "block_decode_ring_kernel"
         launches = run.launches_per_step * args.steps
         step_bytes = w.n_layers * traffic.block_decode_layer_bytes(w.batch, w.heads, w.head_dim, w.ctx_blocks, True)
+    elif args.workload == "dense_decode":
+        run = harness.DenseDecodeStep(w, fill=fill)
+        tokens_per_step = w.batch * w.block_len
+        # a bench step = one CUDA-graph replay of (put the lengths back, then 12 launches, each appending the
+        # block's L_B rows and running its L_B queries); per-launch time = step time / 12
+        run.capture()
+        sampler.start()
+        ms = timed(run.replay, lambda: None, args.steps, args.warmup)
+        clocks = sampler.stop()
+        assert run.status.item() == 0 and (run.cache.len == w.ctx_blocks).all()
+        ms_e2e, h2d, d2h = None, 0, 0
+        alg_bytes = traffic.dense_decode_layer_bytes(w.batch, w.heads, w.head_dim, w.ctx_blocks, w.block_len)
+        dom = "block_decode_mq_kernel"
+        launches = run.launches_per_step * args.steps
+        step_bytes = w.n_layers * alg_bytes
     elif args.workload == "token_decode":
         run = harness.TokenDecodeRun(w, fill=fill)
         tokens_per_step = w.batch
@@ -406,7 +426,7 @@ def main():
     ap.add_argument("--steps", type=int, default=0, help="timed steps (default 200; 3 for the sweep, whose step is a whole generation)")
     ap.add_argument("--warmup", type=int, default=3)
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
-    ap.add_argument("--workload", default="block_decode", choices=["block_decode", "block_decode_16k", "token_decode", "block_prefill", "block_prefill_8k", "sweep"])
+    ap.add_argument("--workload", default="block_decode", choices=["block_decode", "block_decode_16k", "dense_decode", "token_decode", "block_prefill", "block_prefill_8k", "sweep"])
     ap.add_argument("--block-len", type=int, default=4, help="L_B of the generation sweep (1, 2, 4 or 8)")
     ap.add_argument("--prefix-len", type=int, default=0, help="token_decode: prefix length P (default 1 = BASELINE configs[2]; 2 = the paper's main setting)")
     ap.add_argument("--no-cpu-baseline", action="store_true")

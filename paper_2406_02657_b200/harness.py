@@ -145,6 +145,49 @@ class BlockDecodeStep:
             main.wait_event(e)
 
 
+class DenseDecodeStep:
+    """One step of the densified block decoder over all layers (the paper's discussion of future work):
+    per layer one launch appends the block's L_B sub-block rows and runs its L_B queries over the
+    cache.  The caches are pre-filled so that after the append every sequence holds ``ctx_blocks`` rows."""
+
+    def __init__(self, w, device="cuda", fill=None):
+        self.w, self.device = w, device
+        m = w.block_len
+        self.cfg = bt.make_config(w.batch, w.heads, w.head_dim, w.block_len, w.prefix_len, w.max_blocks, w.n_layers)
+        shape = (w.n_layers, w.batch, w.heads, w.max_blocks, w.head_dim)
+        mk = fill if fill is not None else (lambda tid, sh: torch.zeros(sh, dtype=torch.bfloat16, device=device))
+        self.cache = bt.BlockCache(self.cfg, device, k=mk(0, shape), v=mk(1, shape))
+        self.len0 = torch.full((w.n_layers, w.batch), w.ctx_blocks - m, dtype=torch.int32, device=device)
+        self.cache.len.copy_(self.len0)
+        io = (w.n_layers, w.batch, w.heads, m, w.head_dim)
+        self.q, self.k_new, self.v_new = mk(2, io), mk(3, io), mk(4, io)
+        self.out = torch.empty(io, dtype=torch.bfloat16, device=device)
+        self.ws = bt.alloc_workspace(self.cfg, device)
+        self.status = torch.zeros(1, dtype=torch.int32, device=device)
+        self.launches_per_step = w.n_layers
+        self.graph = None
+
+    def rewind(self):
+        self.cache.len.copy_(self.len0, non_blocking=True)
+
+    def step(self):
+        for l in range(self.w.n_layers):
+            bt.bt_block_decode_step_multi(self.cfg, self.cache, l, self.q[l], self.k_new[l], self.v_new[l], self.out[l], self.ws,
+                                          dev_status=self.status)
+
+    def capture(self):
+        self.step()  # anything lazy happens outside the capture
+        self.rewind()
+        torch.cuda.synchronize()
+        self.graph = torch.cuda.CUDAGraph()
+        with torch.cuda.graph(self.graph):
+            self.rewind()
+            self.step()
+
+    def replay(self):
+        self.graph.replay()
+
+
 class TokenDecodeRun:
     """Token-decoder steps over all layers (section 2.4): step 0 of a block resets the local cache and
     appends the P prefix rows (P queries, causal among themselves), step j >= 1 appends the row of the

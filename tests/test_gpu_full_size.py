@@ -78,6 +78,33 @@ def test_block_decode_step_long_context(bt, batch):
             assert_close(run.out[l][seqs][:, :, 0], ref, f"16K-context block decode, batch {batch}, layer {l}")
 
 
+def test_dense_decode_step_full_size(bt):
+    """The densified block decoder at the bench shape: batch 256, 16 heads, 2048 rows after a step that
+    appends 4 rows and runs 4 queries per (sequence, head); two of the 12 layers, twice."""
+    from paper_2406_02657_b200 import harness
+    w = configs.scaled(configs.DENSE_DECODE, n_layers=2)
+    m = w.block_len
+    run = harness.DenseDecodeStep(w, fill=_fill(w))
+    seqs = [0, 101, 255]
+    for _ in range(2):
+        run.rewind()
+        run.out.zero_()
+        torch.cuda.synchronize()
+        before = {l: (gen.torch_to_bits(run.cache.k[l][seqs]), gen.torch_to_bits(run.cache.v[l][seqs])) for l in range(w.n_layers)}
+        run.step()
+        torch.cuda.synchronize()
+        assert run.status.item() == 0 and (run.cache.len == w.ctx_blocks).all()
+        assert torch.equal(run.cache.k[:, :, :, w.ctx_blocks - m:], run.k_new)   # the appended rows, whole batch
+        assert torch.equal(run.cache.v[:, :, :, w.ctx_blocks - m:], run.v_new)
+        for l in range(w.n_layers):
+            c = oracle.Cache(len(seqs), w.heads, w.max_blocks, w.head_dim)
+            c.k[...], c.v[...] = before[l]
+            c.len[...] = w.ctx_blocks - m
+            ref = oracle.block_decode_step_multi(c, *(gen.torch_to_bits(x[l][seqs]) for x in (run.q, run.k_new, run.v_new)))
+            assert_close(run.out[l][seqs], ref, f"full-size dense decode layer {l}", p_bf16=True)
+            assert np.array_equal(gen.torch_to_bits(run.cache.k[l][seqs]), c.k)
+
+
 def test_block_decode_step_through_host_buffers(bt):
     """The e2e path of bench.py: the same step driven from pinned host buffers through
     bt_block_decode_step_host (per-layer calls on several streams) gives the device-resident step's

@@ -44,6 +44,12 @@ BLOCK_DECODE = Workload("block_decode", batch=256, heads=16, head_dim=64, block_
 BLOCK_DECODE_16K = Workload("block_decode_16k", batch=64, heads=16, head_dim=64, block_len=4, prefix_len=1,
                             n_layers=12, max_blocks=4096, ctx_blocks=4096, seed=1012)
 
+# the densified block decoder the paper proposes as future work: a block is L_B sub-block tokens, so the
+# cache holds one row per token (2048 rows for the 2048-token context) and a step appends L_B rows and
+# runs L_B queries
+DENSE_DECODE = Workload("dense_decode", batch=256, heads=16, head_dim=64, block_len=4, prefix_len=1,
+                        n_layers=12, max_blocks=2048, ctx_blocks=2048, seed=1022)
+
 # config 3: token-decoder local decode, 4096 sequences, local cache 1 prefix + up to L_B tokens
 TOKEN_DECODE = Workload("token_decode", batch=4096, heads=16, head_dim=64, block_len=4, prefix_len=1,
                         n_layers=12, max_blocks=1, gen_tokens=4096, seed=1003)
@@ -71,4 +77,4 @@ def scaled(w: Workload, **kw) -> Workload:
     return replace(w, **kw)
 
 
-BY_NAME = {w.name: w for w in (TINY, BLOCK_DECODE, BLOCK_DECODE_16K, TOKEN_DECODE, BLOCK_PREFILL, BLOCK_PREFILL_8K)}
+BY_NAME = {w.name: w for w in (TINY, BLOCK_DECODE, BLOCK_DECODE_16K, DENSE_DECODE, TOKEN_DECODE, BLOCK_PREFILL, BLOCK_PREFILL_8K)}

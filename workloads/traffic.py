@@ -24,6 +24,13 @@ def block_decode_layer_bytes(B: int, H: int, hd: int, ctx_len: int, with_append:
     return kv + qo + app
 
 
+def dense_decode_layer_bytes(B: int, H: int, hd: int, rows_after: int, m: int) -> int:
+    """One layer of one densified block-decoder step: the rows_after - m cached rows (K and V) read,
+    m queries in and m outputs out, the m new K,V rows read once and written once."""
+    row = hd * BF16
+    return B * H * ((rows_after - m) * 2 * row + 2 * m * row + 2 * 2 * m * row)
+
+
 def token_decode_layer_bytes(B: int, H: int, hd: int, rows_before: int, n_new: int = 1) -> int:
     """One layer of one token-decoder step: q, k_new, v_new in; out out; the new rows written
     to the local cache; rows_before cached rows (K and V) read."""
