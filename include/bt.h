@@ -157,8 +157,8 @@ bt_status bt_block_decode_step(const bt_config* cfg, bt_block_cache* cache, int 
  * without room for all n_q rows is left as it is, every query attends over its len[b] rows, and
  * BT_DEV_OVERFLOW is raised.  n_q = 1 computes what bt_block_decode_step computes.
  * Scores and weighted sums run on the tensor cores (bf16 inputs, fp32 accumulation; the softmax
- * weights are rounded to bf16 where they meet V).  Supported: head_dim 64, 1 <= n_q <= 8,
- * N_max >= 32, all pointers 16-byte aligned; otherwise BT_ERR_UNSUPPORTED.  The row range is
+ * weights are rounded to bf16 where they meet V).  Supported: 1 <= n_q <= 8, N_max >= 32, all
+ * pointers 16-byte aligned; otherwise BT_ERR_UNSUPPORTED.  The row range is
  * never split.  workspace: required, as for bt_block_decode_step.
  */
 bt_status bt_block_decode_step_multi(const bt_config* cfg, bt_block_cache* cache, int layer, const void* q,

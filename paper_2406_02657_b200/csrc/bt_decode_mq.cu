@@ -5,8 +5,8 @@
 // queries, which is the point of the proposal.
 //
 // Same streaming structure as the single-query kernel: one persistent CTA per SM, eight warps, every
-// warp on its own with a ring of three 8 KB shared-memory stages (32 K rows + the same 32 V rows)
-// kept full across item boundaries.  What differs is the arithmetic: with m queries per row the work
+// warp on its own with a ring of three 8 KB shared-memory stages (4 KB of K rows + the same V rows:
+// 32 rows at head_dim 64, 16 at 128) kept full across item boundaries.  What differs is the arithmetic: with m queries per row the work
 // is a real [m x hd] x [hd x rows] contraction, m times the single-query flops per byte, which the
 // CUDA cores cannot hide behind the stream - so the stages are filled by TMA tensor copies with the
 // 128-byte swizzle (conflict-free ldmatrix) and scores and weighted sums run on the tensor cores as
@@ -30,9 +30,17 @@ namespace mq {
 constexpr int kWarps = 8;
 constexpr int kThreads = kWarps * 32;
 constexpr int kStages = 3;
-constexpr int ROWS = 32;                       // cache rows per chunk
-constexpr int CHUNK_BYTES = ROWS * 128;        // one TMA box: 64 bf16 x 32 rows
+constexpr int CHUNK_BYTES = 4096;              // K rows of one chunk (and as many bytes of V rows)
 constexpr int STAGE_BYTES = 2 * CHUNK_BYTES;   // K chunk, then V chunk
+// A row is HD/64 TMA boxes of 64 elements (128 bytes, the swizzle span); a chunk holds box after box,
+// each ROWS rows of 128 bytes.
+template <int HD>
+struct Geo {
+    static_assert(HD == 64 || HD == 128, "head_dim must be 64 or 128");
+    static constexpr int NBOX = HD / 64;
+    static constexpr int ROWS = CHUNK_BYTES / (HD * 2);   // cache rows per chunk: 32 or 16
+    static constexpr int BOX_BYTES = ROWS * 128;
+};
 constexpr uint32_t kPollLimit = 1u << 24;      // polls of one wait before giving up (each poll suspends briefly)
 constexpr int kSmemBytes = kWarps * kStages * STAGE_BYTES + kWarps * kStages * 8 + 1024;  // + room to align to 1 KB
 
@@ -70,12 +78,13 @@ __device__ __forceinline__ bool mbar_wait_bounded(uint32_t bar, uint32_t parity)
     return false;
 }
 
-// one box (64 elements x ROWS rows of one slab) global -> shared, completion counted on the mbarrier
-__device__ __forceinline__ void tma_load_box(uint32_t dst, const CUtensorMap* map, uint32_t bar, int row, int slab)
+// one box (64 elements from column `col` x ROWS rows of one slab) global -> shared, completion counted on
+// the mbarrier
+__device__ __forceinline__ void tma_load_box(uint32_t dst, const CUtensorMap* map, uint32_t bar, int col, int row, int slab)
 {
     asm volatile(
         "cp.async.bulk.tensor.3d.shared::cluster.global.tile.mbarrier::complete_tx::bytes [%0], [%1, {%2, %3, %4}], [%5];"
-        ::"r"(dst), "l"(map), "r"(0), "r"(row), "r"(slab), "r"(bar)
+        ::"r"(dst), "l"(map), "r"(col), "r"(row), "r"(slab), "r"(bar)
         : "memory");
 }
 
@@ -111,6 +120,7 @@ struct Work {
     int bh, b, n0, n, nchunks;
     bool append, overflow;
 };
+template <int ROWS>
 __device__ __forceinline__ Work decode_work(int item, const MultiDecodeArgs& a)
 {
     Work w;
@@ -130,7 +140,8 @@ template <int HD>
 __global__ void __launch_bounds__(kThreads, 1)
 block_decode_mq_kernel(const __grid_constant__ CUtensorMap mapK, const __grid_constant__ CUtensorMap mapV, MultiDecodeArgs a)
 {
-    static_assert(HD == 64, "one 64-element box per row");
+    using G = Geo<HD>;
+    constexpr int ROWS = G::ROWS, NBOX = G::NBOX, BOX_BYTES = G::BOX_BYTES;
     extern __shared__ uint8_t smem_raw[];
     const uint32_t base = (smem_u32(smem_raw) + 1023u) & ~1023u;   // the swizzle pattern repeats every 1 KB
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
@@ -161,9 +172,9 @@ block_decode_mq_kernel(const __grid_constant__ CUtensorMap mapK, const __grid_co
     Work pw = {};
     auto p_seek = [&]() {  // move to the next item that has rows; its new rows go into the cache first
         while (p_item < n_items) {
-            pw = decode_work(p_item, a);
+            pw = decode_work<ROWS>(p_item, a);
             if (pw.append) {
-                for (int i = lane; i < a.m * 8; i += 32) {   // 16-byte pieces of the m new K rows and V rows
+                for (int i = lane; i < a.m * (HD / 8); i += 32) {   // 16-byte pieces of the m new K rows and V rows
                     const size_t src = ((size_t)pw.bh * a.m) * HD + (size_t)i * 8;
                     const size_t dst = ((size_t)pw.bh * a.n_max + pw.n0) * HD + (size_t)i * 8;
                     *reinterpret_cast<uint4*>(Kall + dst) = ld_plain(Knew + src);
@@ -188,8 +199,11 @@ block_decode_mq_kernel(const __grid_constant__ CUtensorMap mapK, const __grid_co
             const uint32_t bar = bar0 + 8 * st, dst = ring0 + st * STAGE_BYTES;
             // a box is always delivered whole (rows past the slab arrive as zeros)
             asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(bar), "r"((uint32_t)STAGE_BYTES) : "memory");
-            tma_load_box(dst, &mapK, bar, p_c * ROWS, pw.bh);
-            tma_load_box(dst + CHUNK_BYTES, &mapV, bar, p_c * ROWS, pw.bh);
+#pragma unroll
+            for (int bx = 0; bx < NBOX; ++bx) {
+                tma_load_box(dst + bx * BOX_BYTES, &mapK, bar, bx * 64, p_c * ROWS, pw.bh);
+                tma_load_box(dst + CHUNK_BYTES + bx * BOX_BYTES, &mapV, bar, bx * 64, p_c * ROWS, pw.bh);
+            }
         }
         ++issued;
         if (++p_c == pw.nchunks) {
@@ -202,15 +216,22 @@ block_decode_mq_kernel(const __grid_constant__ CUtensorMap mapK, const __grid_co
 
     // ---- consumer.  Lane (g, t) = (lane / 4, lane % 4) owns query row g and, of every 8 columns, 2t and 2t+1.
     const int g = lane >> 2, t = lane & 3;
-    // lane-constant parts of the ldmatrix addresses: K rows are matrix rows (8 rows x the four 16-byte
-    // pieces 4h..4h+3 per instruction), V rows likewise with .trans (32 rows x one 16-byte piece)
-    uint32_t k_off[2];
+    // Lane-constant parts of the ldmatrix addresses.  16-byte piece p of row r of a chunk lies in box p / 8
+    // at r * 128 + ((p % 8) ^ (r % 8)) * 16.  K: one instruction reads 8 rows x the four pieces 4h..4h+3
+    // (lane = 8 * piece + row).  V, with .trans: at head_dim 64 32 rows x one piece (lane = row); at 128
+    // 16 rows x two neighbouring pieces (lane = 16 * piece + row).
+    constexpr int KH = HD / 32;   // K instructions per 8-row tile
+    uint32_t k_off[KH];
 #pragma unroll
-    for (int h = 0; h < 2; ++h) k_off[h] = (lane & 7) * 128 + ((((h * 4) + (lane >> 3)) ^ (lane & 7)) << 4);
-    const uint32_t v_row = lane * 128;
+    for (int h = 0; h < KH; ++h) {
+        const int p = h * 4 + (lane >> 3);
+        k_off[h] = (p >> 3) * BOX_BYTES + (lane & 7) * 128 + (((p & 7) ^ (lane & 7)) << 4);
+    }
+    const int v_r = HD == 64 ? lane : (lane & 15);        // V row this lane addresses
+    const int v_p = HD == 64 ? 0 : (lane >> 4);           // ... and which piece of the instruction's pair
     bool alive = true;
     for (int item = first; alive && item < n_items; item += stride) {
-        const Work w = decode_work(item, a);
+        const Work w = decode_work<ROWS>(item, a);
         // count this item in on its sequence's counter once its read of the length has returned (the
         // increment is computed from the value read); the result is looked at when the item is done
         int seq_arrival = -1;
@@ -248,34 +269,42 @@ block_decode_mq_kernel(const __grid_constant__ CUtensorMap mapK, const __grid_co
             const int nvalid = min(ROWS, w.n - row_base);
             if (nvalid < ROWS) {
                 // rows past the length may hold anything, and 0 x NaN is NaN: clear their V rows
-                for (int i = lane; i < (ROWS - nvalid) * 8; i += 32)
-                    asm volatile("st.shared.v4.b32 [%0], {%1, %1, %1, %1};" ::"r"(vs + (nvalid + (i >> 3)) * 128 + ((i & 7) << 4)), "r"(0u) : "memory");
+                for (int i = lane; i < NBOX * (ROWS - nvalid) * 8; i += 32) {
+                    const int bx = i / ((ROWS - nvalid) * 8), j = i - bx * ((ROWS - nvalid) * 8);
+                    asm volatile("st.shared.v4.b32 [%0], {%1, %1, %1, %1};" ::"r"(vs + bx * BOX_BYTES + (nvalid + (j >> 3)) * 128 + ((j & 7) << 4)), "r"(0u) : "memory");
+                }
                 asm volatile("fence.proxy.async.shared::cta;" ::: "memory");  // the stage is later rewritten by the copy engine
                 __syncwarp();
             }
-            uint32_t kb[ROWS / 8][2][4], vb[HD / 8][4];
+            constexpr int NV = CHUNK_BYTES / 512;   // V instructions per chunk (512 bytes each)
+            uint32_t kb[ROWS / 8][KH][4], vb[NV][4];
 #pragma unroll
             for (int nt = 0; nt < ROWS / 8; ++nt)
 #pragma unroll
-                for (int h = 0; h < 2; ++h) ldmatrix_x4(ks + nt * 1024 + k_off[h], kb[nt][h]);
+                for (int h = 0; h < KH; ++h) ldmatrix_x4(ks + nt * 1024 + k_off[h], kb[nt][h]);
 #pragma unroll
-            for (int nd = 0; nd < HD / 8; ++nd) ldmatrix_x4_trans(vs + v_row + ((nd ^ (lane & 7)) << 4), vb[nd]);
+            for (int i = 0; i < NV; ++i) {
+                // head_dim 64: piece i of rows 0..31 (k-steps 0 and 1 of column tile i);
+                // head_dim 128: pieces 2i and 2i+1 of rows 0..15 (column tiles 2i and 2i+1)
+                const int p = HD == 64 ? i : 2 * i + v_p;
+                ldmatrix_x4_trans(vs + (p >> 3) * BOX_BYTES + v_r * 128 + (((p & 7) ^ (v_r & 7)) << 4), vb[i]);
+            }
             // the fragments are in registers: hand the stage back and request the next chunk
             ++consumed;
 #pragma unroll
-            for (int nt = 0; nt < ROWS / 8; ++nt) asm volatile("" ::"r"(kb[nt][0][0]), "r"(kb[nt][1][3]) : "memory");
+            for (int nt = 0; nt < ROWS / 8; ++nt) asm volatile("" ::"r"(kb[nt][0][0]), "r"(kb[nt][KH - 1][3]) : "memory");
 #pragma unroll
-            for (int nd = 0; nd < HD / 8; ++nd) asm volatile("" ::"r"(vb[nd][0]), "r"(vb[nd][3]) : "memory");
+            for (int i = 0; i < NV; ++i) asm volatile("" ::"r"(vb[i][0]), "r"(vb[i][3]) : "memory");
             __syncwarp();
             issue_one();
 
-            // S = Q K^T: 4 column tiles of 8 rows, 4 k-steps of 16 dims
+            // S = Q K^T: ROWS / 8 column tiles of 8 rows, HD / 16 k-steps of 16 dims
             float s[ROWS / 8][4];
 #pragma unroll
             for (int nt = 0; nt < ROWS / 8; ++nt) {
                 s[nt][0] = s[nt][1] = s[nt][2] = s[nt][3] = 0.f;
 #pragma unroll
-                for (int h = 0; h < 2; ++h) {
+                for (int h = 0; h < KH; ++h) {
                     mma_rows0to7(s[nt], qa[2 * h][0], qa[2 * h][1], kb[nt][h][0], kb[nt][h][1]);
                     mma_rows0to7(s[nt], qa[2 * h + 1][0], qa[2 * h + 1][1], kb[nt][h][2], kb[nt][h][3]);
                 }
@@ -319,9 +348,15 @@ block_decode_mq_kernel(const __grid_constant__ CUtensorMap mapK, const __grid_co
                 pa[k2][1] = pack_bf16(s[2 * k2 + 1][0], s[2 * k2 + 1][1]);
             }
 #pragma unroll
-            for (int nd = 0; nd < HD / 8; ++nd)
-#pragma unroll
-                for (int k2 = 0; k2 < ROWS / 16; ++k2) mma_rows0to7(o[nd], pa[k2][0], pa[k2][1], vb[nd][2 * k2], vb[nd][2 * k2 + 1]);
+            for (int i = 0; i < NV; ++i) {
+                if constexpr (HD == 64) {
+                    mma_rows0to7(o[i], pa[0][0], pa[0][1], vb[i][0], vb[i][1]);
+                    mma_rows0to7(o[i], pa[1][0], pa[1][1], vb[i][2], vb[i][3]);
+                } else {
+                    mma_rows0to7(o[2 * i], pa[0][0], pa[0][1], vb[i][0], vb[i][1]);
+                    mma_rows0to7(o[2 * i + 1], pa[0][0], pa[0][1], vb[i][2], vb[i][3]);
+                }
+            }
         }
         if (!alive) break;
         float l = l_run;
@@ -358,11 +393,12 @@ block_decode_mq_kernel(const __grid_constant__ CUtensorMap mapK, const __grid_co
 bool multi_decode_supported(const MultiDecodeArgs& a)
 {
     auto al = [](const void* p) { return (reinterpret_cast<uintptr_t>(p) & 15u) == 0; };
-    return a.hd == 64 && a.m >= 1 && a.m <= 8 && a.n_max >= mq::ROWS && al(a.q) && al(a.k) && al(a.v) && al(a.k_new) && al(a.v_new) && al(a.out) &&
+    return (a.hd == 64 || a.hd == 128) && a.m >= 1 && a.m <= 8 && a.n_max >= 32 && al(a.q) && al(a.k) && al(a.v) && al(a.k_new) && al(a.v_new) && al(a.out) &&
            tensor_map_encode_fn() != nullptr;
 }
 
-cudaError_t launch_block_decode_multi(const MultiDecodeArgs& a, cudaStream_t stream)
+template <int HD>
+static cudaError_t launch_multi_t(const MultiDecodeArgs& a, cudaStream_t stream)
 {
     using namespace mq;
     constexpr int kMaxDevices = 64;
@@ -372,7 +408,7 @@ cudaError_t launch_block_decode_multi(const MultiDecodeArgs& a, cudaStream_t str
     if (e != cudaSuccess) return e;
     if (dev < 0 || dev >= kMaxDevices) return cudaErrorInvalidDevice;
     if (!sm_count[dev]) {
-        e = cudaFuncSetAttribute(block_decode_mq_kernel<64>, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemBytes);
+        e = cudaFuncSetAttribute(block_decode_mq_kernel<HD>, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemBytes);
         if (e != cudaSuccess) return e;
         int n = 0;
         e = cudaDeviceGetAttribute(&n, cudaDevAttrMultiProcessorCount, dev);
@@ -382,10 +418,16 @@ cudaError_t launch_block_decode_multi(const MultiDecodeArgs& a, cudaStream_t str
     const long long items = (long long)a.B * a.H;
     if (items > 0x7fffffffLL - 4096) return cudaErrorInvalidConfiguration;
     CUtensorMap mk, mv;
-    if (!make_slab_map(&mk, a.k, 64, a.n_max, a.n_max, items, ROWS) || !make_slab_map(&mv, a.v, 64, a.n_max, a.n_max, items, ROWS))
+    if (!make_slab_map(&mk, a.k, HD, a.n_max, a.n_max, items, Geo<HD>::ROWS) ||
+        !make_slab_map(&mv, a.v, HD, a.n_max, a.n_max, items, Geo<HD>::ROWS))
         return cudaErrorInvalidValue;
     const long long grid = items < sm_count[dev] ? items : sm_count[dev];
-    return launch_pdl(block_decode_mq_kernel<64>, dim3((unsigned)grid), dim3(kThreads), (size_t)kSmemBytes, stream, mk, mv, a);
+    return launch_pdl(block_decode_mq_kernel<HD>, dim3((unsigned)grid), dim3(kThreads), (size_t)kSmemBytes, stream, mk, mv, a);
+}
+
+cudaError_t launch_block_decode_multi(const MultiDecodeArgs& a, cudaStream_t stream)
+{
+    return a.hd == 64 ? launch_multi_t<64>(a, stream) : launch_multi_t<128>(a, stream);
 }
 
 }  // namespace bt

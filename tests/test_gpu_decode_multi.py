@@ -24,14 +24,15 @@ def rnd(seed, tid, shape):
     return gen.normal_bf16_bits(seed, tid, shape)
 
 
+@pytest.mark.parametrize("hd", [64, 128])
 @pytest.mark.parametrize("m", [1, 2, 4, 8])
-def test_multi_step_ragged_lengths_three_steps(bt, m):
+def test_multi_step_ragged_lengths_three_steps(bt, m, hd):
     """Lengths around every chunk boundary, an empty cache, caches with exactly room, one row short of
     room and full; rows past each length hold NaN; three steps in a row on one workspace."""
-    B, H, hd, N = 10, 3, 64, 168
+    B, H, N = 12, 3, 168
     cfg = bt.make_config(B, H, hd, m, 1, N, 1)
-    lens = np.array([0, 1, 31, 32, 33, 95, N - 3 * m, N - m, N - m + 1, N], np.int32)
-    k, v = rnd(400 + m, 1, (B, H, N, hd)), rnd(400 + m, 2, (B, H, N, hd))
+    lens = np.array([0, 1, 15, 16, 31, 32, 33, 95, N - 3 * m, N - m, N - m + 1, N], np.int32)
+    k, v = rnd(400 + m + hd, 1, (B, H, N, hd)), rnd(400 + m + hd, 2, (B, H, N, hd))
     oc = oracle.Cache(B, H, N, hd)
     oc.k[...], oc.v[...], oc.len[...] = k, v, lens
     kp, vp = k.copy(), v.copy()
@@ -45,7 +46,7 @@ def test_multi_step_ragged_lengths_three_steps(bt, m):
     ws = bt.alloc_workspace(cfg)
     out = torch.empty((B, H, m, hd), dtype=torch.bfloat16, device="cuda")
     for step in range(3):
-        q, kn, vn = (rnd(410 + m, 3 * step + i, (B, H, m, hd)) for i in range(3))
+        q, kn, vn = (rnd(410 + m + hd, 3 * step + i, (B, H, m, hd)) for i in range(3))
         st = status_word()
         out.fill_(7.0)
         bt.bt_block_decode_step_multi(cfg, cache, 0, to_dev(q), to_dev(kn), to_dev(vn), out, ws, dev_status=st)
@@ -53,7 +54,7 @@ def test_multi_step_ragged_lengths_three_steps(bt, m):
         ref = oracle.block_decode_step_multi(oc, q, kn, vn)
         assert cache.len[0].cpu().tolist() == oc.len.tolist(), f"step {step}: lengths"
         assert st.item() == int(oc.status[0]) and st.item() & bt.BT_DEV_OVERFLOW  # the full cache at least
-        assert_close(out, ref, f"multi step {step} m={m}", p_bf16=True)
+        assert_close(out, ref, f"multi step {step} m={m} hd={hd}", p_bf16=True)
         gk, gv = gen.torch_to_bits(cache.k[0]), gen.torch_to_bits(cache.v[0])
         for b in range(B):
             n = int(oc.len[b])
@@ -62,10 +63,11 @@ def test_multi_step_ragged_lengths_three_steps(bt, m):
     assert not ws.view(torch.int32)[-(B * H + B):].any()   # the arrival counters are back at zero
 
 
-def test_multi_step_causal_rule_among_the_new_rows(bt):
+@pytest.mark.parametrize("hd,n0", [(64, 45), (128, 45), (64, 62), (128, 14)])
+def test_multi_step_causal_rule_among_the_new_rows(bt, hd, n0):
     """New row j carries a key that dominates everything: query i must return the value of the last
-    new row it may see (row i), never a later one."""
-    B, H, hd, N, m, n0 = 2, 2, 64, 128, 4, 45
+    new row it may see (row i), never a later one.  (n0 = 62 and 14: the new rows straddle a chunk end.)"""
+    B, H, N, m = 2, 2, 128, 4
     cfg = bt.make_config(B, H, hd, m, 1, N, 1)
     cache = bt.BlockCache(cfg)
     cache.k[0].copy_(to_dev(rnd(420, 1, (B, H, N, hd))))
@@ -75,7 +77,7 @@ def test_multi_step_causal_rule_among_the_new_rows(bt):
     kn = np.zeros((B, H, m, hd), np.float32)
     vn = np.zeros((B, H, m, hd), np.float32)
     for j in range(m):
-        kn[:, :, j] = 6.0 + 3.0 * j            # later rows dominate earlier ones by e^(2*64*3/8) each
+        kn[:, :, j] = 6.0 + 3.0 * j            # later rows dominate earlier ones by e^(2*3*sqrt(hd)) each
         vn[:, :, j] = np.arange(hd) - 30.0 + 100.0 * j
     out = torch.empty((B, H, m, hd), dtype=torch.bfloat16, device="cuda")
     bt.bt_block_decode_step_multi(cfg, cache, 0, to_dev(q), to_dev(gen.f32_to_bf16_bits(kn)), to_dev(gen.f32_to_bf16_bits(vn)),
@@ -132,7 +134,7 @@ def test_multi_step_many_items_per_warp_and_single_query_entry_points_agree(bt):
 
 def test_multi_step_rejects_what_it_does_not_support(bt):
     x = torch.zeros((2, 2, 4, 128), dtype=torch.bfloat16, device="cuda")
-    cfg = bt.make_config(2, 2, 128, 4, 1, 64, 1)
+    cfg = bt.make_config(2, 2, 128, 4, 1, 24, 1)   # a cache shorter than one chunk
     with pytest.raises(bt.BtError) as e:
         bt.bt_block_decode_step_multi(cfg, bt.BlockCache(cfg), 0, x, x, x, torch.empty_like(x), bt.alloc_workspace(cfg))
     assert "BT_ERR_UNSUPPORTED" in str(e.value)
