@@ -76,6 +76,39 @@ def test_block_path_touches_nothing_outside_its_rows(bt):
         assert st.item() == bt.BT_DEV_OVERFLOW == int(oc.status[0])
 
 
+@pytest.mark.parametrize("hd", [64, 128])
+def test_multi_query_step_touches_nothing_outside_its_rows(bt, hd):
+    rng = np.random.default_rng(11)
+    B, H, N, m = 23, 5, 80, 4
+    cfg = bt.make_config(B, H, hd, m, 1, N, 1)
+    k, v = Guarded((1, B, H, N, hd), torch.bfloat16), Guarded((1, B, H, N, hd), torch.bfloat16)
+    ln = Guarded((1, B), torch.int32)
+    q, kn, vn, out = (Guarded((B, H, m, hd), torch.bfloat16) for _ in range(4))
+    ws = Guarded((max(bt.bt_workspace_bytes(cfg), 4) // 4,), torch.float32)
+    bt.bt_workspace_init(cfg, ws.t)
+    lens = rng.integers(0, N + 1, B).astype(np.int32)
+    lens[0], lens[1], lens[2] = 0, N, N - m + 1   # empty; full; one row short of room for the m rows
+    kb, vb = gen.normal_bf16_bits(500 + hd, 1, (B, H, N, hd)), gen.normal_bf16_bits(500 + hd, 2, (B, H, N, hd))
+    k.t[0].copy_(to_dev(kb)); v.t[0].copy_(to_dev(vb)); ln.t[0].copy_(torch.from_numpy(lens).cuda())
+    qb, knb, vnb = (gen.normal_bf16_bits(500 + hd, 3 + i, (B, H, m, hd)) for i in range(3))
+    q.t.copy_(to_dev(qb)); kn.t.copy_(to_dev(knb)); vn.t.copy_(to_dev(vnb))
+    cache = bt.BlockCache(cfg, k=k.t, v=v.t, length=ln.t)
+    st = status_word()
+    bt.bt_block_decode_step_multi(cfg, cache, 0, q.t, kn.t, vn.t, out.t, ws.t, dev_status=st)
+    torch.cuda.synchronize()
+    oc = oracle.Cache(B, H, N, hd)
+    oc.k[...], oc.v[...], oc.len[...] = kb, vb, lens
+    ref = oracle.block_decode_step_multi(oc, qb, knb, vnb)
+    for g in (k, v, ln, q, kn, vn, out, ws):
+        assert g.guards_intact()
+    # the cache differs from before only in the appended rows; lengths advanced except where there was no room
+    assert np.array_equal(gen.torch_to_bits(k.t[0]), oc.k) and np.array_equal(gen.torch_to_bits(v.t[0]), oc.v)
+    assert np.array_equal(ln.t[0].cpu().numpy(), oc.len) and oc.len[1] == N and oc.len[2] == N - m + 1 and oc.len[0] == m
+    assert np.array_equal(gen.torch_to_bits(q.t), qb) and np.array_equal(gen.torch_to_bits(kn.t), knb)
+    assert_close(out.t, ref, f"guarded multi-query step hd={hd}", p_bf16=True)
+    assert st.item() == bt.BT_DEV_OVERFLOW == int(oc.status[0])
+
+
 def test_token_step_touches_nothing_outside_its_rows(bt):
     rng = np.random.default_rng(11)
     B, H, hd, L_B, P = 53, 16, 64, 4, 1
