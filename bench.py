@@ -197,7 +197,7 @@ def workload_config(w, name):
     c = {"workload": name, "batch": w.batch, "heads": w.heads, "head_dim": w.head_dim, "block_len": w.block_len,
          "prefix_len": w.prefix_len, "n_layers": w.n_layers}
     if name == "block_decode":
-        c.update(workload="block_decode: BASELINE configs[1], per layer append 1 block row then attend over 512 rows",
+        c.update(workload="block_decode: benchmark configs[1], per layer append 1 block row then attend over 512 rows",
                  ctx_blocks=w.ctx_blocks, context_tokens=w.ctx_blocks * w.block_len,
                  l2="no flush: 6.4 GB of KV per step, 537 MB per launch, L2 is 126 MB")
     elif name == "block_decode_16k":
@@ -211,10 +211,10 @@ def workload_config(w, name):
                  ctx_rows=w.ctx_blocks, context_tokens=w.ctx_blocks,
                  l2="no flush: 2.1 GB of KV per launch")
     elif name == "token_decode":
-        c.update(workload="token_decode: BASELINE configs[2], fused reset+append+local attention, 12 launches per token step",
+        c.update(workload="token_decode: benchmark configs[2], fused reset+append+local attention, 12 launches per token step",
                  l2="no flush: inputs rotate over a ring larger than L2")
     elif name == "sweep":
-        c.update(workload=f"sweep: BASELINE configs[4], decode-heavy generation at L_B = {w.block_len}: prompt {w.prompt_tokens} tokens, "
+        c.update(workload=f"sweep: benchmark configs[4], decode-heavy generation at L_B = {w.block_len}: prompt {w.prompt_tokens} tokens, "
                           f"{w.gen_tokens} generated, block step every L_B tokens and token step every token",
                  prompt_tokens=w.prompt_tokens, gen_tokens=w.gen_tokens, max_blocks=w.max_blocks,
                  l2="no flush: the block cache alone is far larger than L2")
@@ -222,7 +222,7 @@ def workload_config(w, name):
         c.update(workload="block_prefill_8k: the 8K-prompt case (2048 prompt blocks at L_B = 4, batch 8), same path as configs[3]",
                  prompt_blocks=w.prompt_blocks, l2="no flush: 3.2 GB of Q,K,V,out per step")
     elif name == "block_prefill":
-        c.update(workload="block_prefill: BASELINE configs[3], dense causal attention over 512 prompt blocks",
+        c.update(workload="block_prefill: benchmark configs[3], dense causal attention over 512 prompt blocks",
                  prompt_blocks=w.prompt_blocks, l2="no flush: 3.2 GB of Q,K,V,out per step")
     return c
 
@@ -430,7 +430,7 @@ def main():
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--workload", default="block_decode", choices=["block_decode", "block_decode_16k", "dense_decode", "token_decode", "block_prefill", "block_prefill_8k", "sweep"])
     ap.add_argument("--block-len", type=int, default=4, help="L_B of the generation sweep (1, 2, 4 or 8)")
-    ap.add_argument("--prefix-len", type=int, default=0, help="token_decode: prefix length P (default 1 = BASELINE configs[2]; 2 = the paper's main setting)")
+    ap.add_argument("--prefix-len", type=int, default=0, help="token_decode: prefix length P (default 1 = benchmark configs[2]; 2 = the paper's main setting)")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--batch", type=int, default=0, help="override the batch (profiling a small case; not a bench number)")
     ap.add_argument("--layers", type=int, default=0, help="override the layer count (profiling a small case)")

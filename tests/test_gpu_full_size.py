@@ -27,7 +27,7 @@ def _fill(w):
 
 
 def test_block_decode_step_full_size(bt):
-    """BASELINE configs[1]: batch 256, 16 heads, head_dim 64, 512 rows after the append, 12 layers."""
+    """benchmark configs[1]: batch 256, 16 heads, head_dim 64, 512 rows after the append, 12 layers."""
     from paper_2406_02657_b200 import harness
     w = configs.BLOCK_DECODE
     run = harness.BlockDecodeStep(w, fill=_fill(w))
@@ -126,7 +126,7 @@ def test_block_decode_step_through_host_buffers(bt):
 
 
 def test_token_decode_full_size_two_blocks(bt):
-    """BASELINE configs[2]: 4096 sequences, 12 layers, local cache 1 prefix + up to L_B rows; two
+    """benchmark configs[2]: 4096 sequences, 12 layers, local cache 1 prefix + up to L_B rows; two
     blocks of consecutive token steps, lengths against the integer schedule model at full size."""
     from paper_2406_02657_b200 import harness
     w = configs.TOKEN_DECODE
@@ -182,7 +182,7 @@ def test_token_decode_full_batch_prefix_length_two(bt):
 
 
 def test_block_prefill_full_size(bt):
-    """BASELINE configs[3]: batch 32, 512 prompt blocks, 16 heads, head_dim 128, 12 layers."""
+    """benchmark configs[3]: batch 32, 512 prompt blocks, 16 heads, head_dim 128, 12 layers."""
     from paper_2406_02657_b200 import harness
     w = configs.BLOCK_PREFILL
     run = harness.PrefillRun(w, fill=_fill(w))

@@ -1,4 +1,4 @@
-"""Decode-heavy generation (BASELINE configs[4]: the L_B sweep) through the harness driver: every
+"""Decode-heavy generation (benchmark configs[4]: the L_B sweep) through the harness driver: every
 token step and block step of a small generation against the oracle at L_B = 1, 2, 4, 8, and the
 full-size run (batch 512, prompt 128, 2048 generated tokens) at L_B = 4 with lengths, cache rows and
 sampled outputs checked."""
