@@ -22,6 +22,7 @@
 
 #include "bt_common.cuh"
 #include "bt_kernels.h"
+#include "bt_mbarrier.cuh"
 #include "bt_tensor_map.h"
 
 namespace bt {
@@ -44,39 +45,7 @@ struct Geo {
 constexpr uint32_t kPollLimit = 1u << 24;      // polls of one wait before giving up (each poll suspends briefly)
 constexpr int kSmemBytes = kWarps * kStages * STAGE_BYTES + kWarps * kStages * 8 + 1024;  // + room to align to 1 KB
 
-__device__ __forceinline__ uint32_t smem_u32(const void* p) { return (uint32_t)__cvta_generic_to_shared(p); }
-
-__device__ __forceinline__ bool mbar_test_wait(uint32_t bar, uint32_t parity)
-{
-    uint32_t ok;
-    asm volatile(
-        "{\n\t.reg .pred p;\n\t"
-        "mbarrier.test_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
-        "selp.u32 %0, 1, 0, p;\n\t}"
-        : "=r"(ok)
-        : "r"(bar), "r"(parity)
-        : "memory");
-    return ok != 0;
-}
-__device__ __forceinline__ bool mbar_try_wait(uint32_t bar, uint32_t parity)
-{
-    uint32_t ok;
-    asm volatile(
-        "{\n\t.reg .pred p;\n\t"
-        "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
-        "selp.u32 %0, 1, 0, p;\n\t}"
-        : "=r"(ok)
-        : "r"(bar), "r"(parity)
-        : "memory");
-    return ok != 0;
-}
-__device__ __forceinline__ bool mbar_wait_bounded(uint32_t bar, uint32_t parity)
-{
-    if (mbar_test_wait(bar, parity)) return true;
-    for (uint32_t it = 0; it < kPollLimit; ++it)
-        if (mbar_try_wait(bar, parity)) return true;
-    return false;
-}
+__device__ __forceinline__ bool mbar_wait_bounded(uint32_t bar, uint32_t parity) { return mbar_wait_polls(bar, parity, kPollLimit); }
 
 // one box (64 elements from column `col` x ROWS rows of one slab) global -> shared, completion counted on
 // the mbarrier
@@ -150,7 +119,7 @@ block_decode_mq_kernel(const __grid_constant__ CUtensorMap mapK, const __grid_co
 
     if (lane == 0) {
         for (int s = 0; s < kStages; ++s)
-            asm volatile("mbarrier.init.shared::cta.b64 [%0], 1;" ::"r"(bar0 + 8 * s) : "memory");
+            mbar_init(bar0 + 8 * s, 1);
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
         asm volatile("prefetch.tensormap [%0];" ::"l"(&mapK) : "memory");
         asm volatile("prefetch.tensormap [%0];" ::"l"(&mapV) : "memory");
@@ -198,7 +167,7 @@ block_decode_mq_kernel(const __grid_constant__ CUtensorMap mapK, const __grid_co
         if (lane == 0) {
             const uint32_t bar = bar0 + 8 * st, dst = ring0 + st * STAGE_BYTES;
             // a box is always delivered whole (rows past the slab arrive as zeros)
-            asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(bar), "r"((uint32_t)STAGE_BYTES) : "memory");
+            mbar_expect_tx(bar, (uint32_t)STAGE_BYTES);
 #pragma unroll
             for (int bx = 0; bx < NBOX; ++bx) {
                 tma_load_box(dst + bx * BOX_BYTES, &mapK, bar, bx * 64, p_c * ROWS, pw.bh);

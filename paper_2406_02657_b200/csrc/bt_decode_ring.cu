@@ -20,6 +20,7 @@
 // every item has read the old one.  Both counters return to zero before the kernel ends.
 #include "bt_common.cuh"
 #include "bt_kernels.h"
+#include "bt_mbarrier.cuh"
 
 namespace bt {
 namespace ring {
@@ -50,40 +51,7 @@ struct Geo {
 template <int HD>
 constexpr int smem_bytes() { return kWarps * kStages * Geo<HD>::STAGE_BYTES + kWarps * kStages * 8; }
 
-__device__ __forceinline__ uint32_t smem_u32(const void* p) { return (uint32_t)__cvta_generic_to_shared(p); }
-
-__device__ __forceinline__ bool mbar_try_wait(uint32_t bar, uint32_t parity)
-{
-    uint32_t ok;
-    asm volatile(
-        "{\n\t.reg .pred p;\n\t"
-        "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
-        "selp.u32 %0, 1, 0, p;\n\t}"
-        : "=r"(ok)
-        : "r"(bar), "r"(parity)
-        : "memory");
-    return ok != 0;
-}
-// Non-blocking test: far cheaper than try_wait when the copy has already landed (the usual case).
-__device__ __forceinline__ bool mbar_test_wait(uint32_t bar, uint32_t parity)
-{
-    uint32_t ok;
-    asm volatile(
-        "{\n\t.reg .pred p;\n\t"
-        "mbarrier.test_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
-        "selp.u32 %0, 1, 0, p;\n\t}"
-        : "=r"(ok)
-        : "r"(bar), "r"(parity)
-        : "memory");
-    return ok != 0;
-}
-__device__ __forceinline__ bool mbar_wait_bounded(uint32_t bar, uint32_t parity)
-{
-    if (mbar_test_wait(bar, parity)) return true;
-    for (uint32_t it = 0; it < kPollLimit; ++it)
-        if (mbar_try_wait(bar, parity)) return true;
-    return false;
-}
+__device__ __forceinline__ bool mbar_wait_bounded(uint32_t bar, uint32_t parity) { return mbar_wait_polls(bar, parity, kPollLimit); }
 // bytes global -> shared, completion counted on the mbarrier; the rows are read once, so they are
 // marked evict-first in L2
 __device__ __forceinline__ void bulk_load(uint32_t dst, const void* src, uint32_t bytes, uint32_t bar, uint64_t policy)
@@ -143,7 +111,7 @@ __global__ void __launch_bounds__(kThreads, 1) block_decode_ring_kernel(DecodeAr
 
     if (lane == 0) {
         for (int s = 0; s < kStages; ++s)
-            asm volatile("mbarrier.init.shared::cta.b64 [%0], 1;" ::"r"(bar0 + 8 * s) : "memory");
+            mbar_init(bar0 + 8 * s, 1);
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     }
     __syncwarp();
@@ -196,7 +164,7 @@ __global__ void __launch_bounds__(kThreads, 1) block_decode_ring_kernel(DecodeAr
         if (lane == 0) {
             const uint32_t bar = bar0 + 8 * st, dst = ring0 + st * G::STAGE_BYTES;
             const size_t off = ((size_t)pw.bh * a.n_max + row) * HD;
-            asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(bar), "r"(2 * bytes) : "memory");
+            mbar_expect_tx(bar, 2 * bytes);
             bulk_load(dst, Kall + off, bytes, bar, policy);
             bulk_load(dst + G::CHUNK_BYTES, Vall + off, bytes, bar, policy);
         }
