@@ -38,6 +38,7 @@ constexpr int kWarps = BT_DEC_WARPS;
 constexpr int kThreads = kWarps * 32;
 constexpr int kStages = BT_DEC_STAGES;
 constexpr int kUnroll = BT_DEC_UNROLL;     // rows per lane group per chunk
+constexpr int kPrefetchChunks = 16;         // chunks of a warp's first item warmed in L2 ahead of the dependent-launch wait
 constexpr uint32_t kPollLimit = 1u << 24;  // polls of one wait before giving up (each poll suspends briefly)
 
 template <int HD>
@@ -124,22 +125,24 @@ __global__ void __launch_bounds__(kThreads, 1) block_decode_ring_kernel(DecodeAr
     const int first = warp * gridDim.x + blockIdx.x;   // neighbouring items go to different SMs
     bf16* Kall = reinterpret_cast<bf16*>(a.k);
     bf16* Vall = reinterpret_cast<bf16*>(a.v);
-    // While the kernel before this one drains, warm L2 with the first ring-full of this warp's first
-    // item (rows 0.. of its slab, whatever its length turns out to be: the rows exist either way), its
-    // length and its query.  A prefetch returns nothing to the thread, so it is safe ahead of the wait.
+    // While the kernel before this one drains, warm L2 with this warp's first item (up to kPrefetchChunks
+    // chunks of it), its length and its query: CTAs that are placed early sit idle until the last CTA
+    // of the previous kernel is gone, and HBM is not busy during that tail.  A prefetch returns nothing
+    // to the thread, so it is safe ahead of the wait.  How many rows to touch comes from a look at the
+    // length that may be out of date (read past L1, so that no stale copy stays behind for the read
+    // after the wait): it is only a hint for the prefetch and never decides what is computed.
     if (first < n_items && a.splits == 1) {
+        int n_hint = __ldcg(a.len + first / a.H);
+        n_hint = n_hint < 0 ? 0 : (n_hint >= a.n_max ? a.n_max : n_hint + 1);
         const size_t off = (size_t)first * a.n_max * HD;
-        const int lines = min(kStages * G::CHUNK_BYTES, a.n_max * G::ROW_BYTES) / 128;  // 128-byte lines to touch
+        const int lines = (min(kPrefetchChunks * G::CHUNK_BYTES, n_hint * G::ROW_BYTES) + 127) / 128;  // 128-byte lines to touch
         for (int i = lane; i < lines; i += 32) {
             asm volatile("prefetch.global.L2 [%0];" ::"l"(reinterpret_cast<const char*>(Kall + off) + (size_t)i * 128));
             asm volatile("prefetch.global.L2 [%0];" ::"l"(reinterpret_cast<const char*>(Vall + off) + (size_t)i * 128));
         }
-        if (lane == 0) {
-            asm volatile("prefetch.global.L2 [%0];" ::"l"(a.len + first / a.H));
-            asm volatile("prefetch.global.L2 [%0];" ::"l"(reinterpret_cast<const bf16*>(a.q) + (size_t)first * HD));
-        }
+        if (lane == 0) asm volatile("prefetch.global.L2 [%0];" ::"l"(reinterpret_cast<const bf16*>(a.q) + (size_t)first * HD));
     }
-    pdl_wait();  // nothing above read or wrote global memory
+    pdl_wait();  // nothing above wrote global memory, or used a value read from it for more than a prefetch hint
 
     // ---- producer cursor (kept by every lane, acted on by lane 0): next chunk to request
     int p_item = first, p_c = 0, p_nchunks = 0;
