@@ -42,6 +42,7 @@ struct Geo {
     static constexpr int ROWS = CHUNK_BYTES / (HD * 2);   // cache rows per chunk: 32 or 16
     static constexpr int BOX_BYTES = ROWS * 128;
 };
+constexpr int kPrefetchChunks = 16;            // chunks of a warp's first item warmed in L2 ahead of the dependent-launch wait
 constexpr uint32_t kPollLimit = 1u << 24;      // polls of one wait before giving up (each poll suspends briefly)
 constexpr int kSmemBytes = kWarps * kStages * STAGE_BYTES + kWarps * kStages * 8 + 1024;  // + room to align to 1 KB
 
@@ -126,13 +127,27 @@ block_decode_mq_kernel(const __grid_constant__ CUtensorMap mapK, const __grid_co
     }
     __syncwarp();
     pdl_launch_dependents();
-    pdl_wait();  // nothing above touched global memory
 
     const int n_items = a.B * a.H;
     const int stride = kWarps * gridDim.x;
     const int first = warp * gridDim.x + blockIdx.x;   // neighbouring items go to different SMs
     bf16* Kall = reinterpret_cast<bf16*>(a.k);
     bf16* Vall = reinterpret_cast<bf16*>(a.v);
+    // While the kernel before this one drains, warm L2 with the start of this warp's first item (CTAs
+    // placed early sit idle until the previous kernel's last CTA is gone, and HBM is not busy in that
+    // tail).  A prefetch returns nothing to the thread, so it is safe ahead of the wait; the row count
+    // comes from a look at the length that may be out of date (read past L1) and is only a hint.
+    if (first < n_items) {
+        int n_hint = __ldcg(a.len + first / a.H);
+        n_hint = n_hint < 0 ? 0 : (n_hint > a.n_max ? a.n_max : n_hint);
+        const size_t off = (size_t)first * a.n_max * HD;
+        const int lines = (min(kPrefetchChunks * CHUNK_BYTES, n_hint * HD * 2) + 127) / 128;
+        for (int i = lane; i < lines; i += 32) {
+            asm volatile("prefetch.global.L2 [%0];" ::"l"(reinterpret_cast<const char*>(Kall + off) + (size_t)i * 128));
+            asm volatile("prefetch.global.L2 [%0];" ::"l"(reinterpret_cast<const char*>(Vall + off) + (size_t)i * 128));
+        }
+    }
+    pdl_wait();  // nothing above wrote global memory, or used a value read from it for more than a prefetch hint
     const bf16* Knew = reinterpret_cast<const bf16*>(a.k_new);
     const bf16* Vnew = reinterpret_cast<const bf16*>(a.v_new);
 
