@@ -87,3 +87,35 @@ def test_mutant_is_caught(name, tmp_path, monkeypatch):
 def test_unmutated_source_passes_the_same_pins():
     for f in PIN_FUNCS:
         f()
+
+
+# The densified block-decoder step is written in the oracle's Python layer (append, then one plain decode
+# per query over a growing prefix): its planted mistakes are edits of that source, run against the pins
+# that compare it with dense causal attention.
+PY_MUTANTS = {
+    "multi_query_sees_one_row_less": ("before + i + 1, before)", "before + i, before)"),
+    "multi_query_sees_one_row_more": ("before + i + 1, before)", "np.minimum(before + i + 2, after), before)"),
+    "multi_query_not_causal": ("before + i + 1, before)", "after, before)"),
+    "multi_query_outputs_shifted": ("out[:, :, i] = block_decode_attn(c, np.ascontiguousarray(q[:, :, i])",
+                                    "out[:, :, i] = block_decode_attn(c, np.ascontiguousarray(q[:, :, (i + 1) % m])"),
+    "multi_query_rows_not_appended": ("    kv_append(c, k_new, v_new)\n    after = c.len.copy()", "    after = c.len.copy()"),
+}
+
+
+@pytest.mark.parametrize("name", sorted(PY_MUTANTS))
+def test_python_layer_mutant_is_caught(name, monkeypatch):
+    old, new = PY_MUTANTS[name]
+    path = oracle.__file__
+    src = open(path).read()
+    assert src.count(old) == 1, f"mutation site for {name} not found"
+    ns = {"__name__": "oracle", "__file__": path, "__package__": "oracle"}
+    exec(compile(src.replace(old, new), path, "exec"), ns)
+    monkeypatch.setattr(oracle, "block_decode_step_multi", ns["block_decode_step_multi"])
+    caught = []
+    for f in (pins.test_densified_step_is_the_matching_rows_of_dense_causal_attention,
+              pins.test_densified_step_without_room_appends_nothing):
+        try:
+            f()
+        except AssertionError:
+            caught.append(f.__name__)
+    assert caught, f"no pin noticed the planted mistake '{name}'"
