@@ -36,11 +36,15 @@ float scale_log2(const bt_config* c)
 int choose_splits(const bt_config* c)
 {
     if (c->decode_splits > 0) return c->decode_splits;
-    // enough CTAs for a few per SM; never fewer than 16 rows per split
+    // enough work items to reach every SM several times over, each of at least 128 rows (four chunks of the
+    // streaming kernel; below that the per-item costs show) - short caches may still be cut into up to 4
+    // parts of at least 16 rows
     const long long bh = (long long)c->batch * c->heads;
-    const long long target = 148 * 4;
+    const long long target = 512;
     long long s = (target + bh - 1) / bh;
-    long long by_rows = c->max_blocks / 16;
+    long long by_rows = c->max_blocks / 128;
+    const long long small = c->max_blocks / 16 < 4 ? c->max_blocks / 16 : 4;
+    if (by_rows < small) by_rows = small;
     if (by_rows < 1) by_rows = 1;
     if (s > by_rows) s = by_rows;
     if (s > 32) s = 32;

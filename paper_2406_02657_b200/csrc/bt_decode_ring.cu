@@ -87,7 +87,9 @@ __device__ __forceinline__ Work decode_work(int item, const DecodeArgs& a)
     w.overflow = a.k_new != nullptr && !append;
     n += append ? 1 : 0;
     w.n = n;
-    const int per = (n + a.splits - 1) / a.splits;
+    // rows per split, rounded up to whole 32-row groups so that every split starts on a chunk boundary
+    // (trailing splits may then be empty)
+    const int per = a.splits == 1 ? n : (((n + a.splits - 1) / a.splits + 31) & ~31);
     w.r0 = min(n, w.sp * per);
     const int r1 = min(n, w.r0 + per);
     w.new_row = append && r1 == n && w.r0 < n;   // exactly one split ends at row n-1
