@@ -145,6 +145,23 @@ class BlockDecodeStep:
             main.wait_event(e)
 
 
+    def capture_host(self, n_streams=3):
+        """Capture rewind + step_host (the copies from and to pinned host memory included) into a CUDA graph,
+        so that a step costs the host one launch instead of some sixty API calls; replay_host() runs it."""
+        self._host_buffers()
+        self.rewind()
+        self.step_host(n_streams)   # creates the side streams, their workspaces and events outside the capture
+        self.rewind()
+        torch.cuda.synchronize()
+        self.graph_host = torch.cuda.CUDAGraph()
+        with torch.cuda.graph(self.graph_host):
+            self.rewind()
+            self.step_host(n_streams)
+
+    def replay_host(self):
+        self.graph_host.replay()
+
+
 class DenseDecodeStep:
     """One step of the densified block decoder over all layers (the paper's discussion of future work):
     per layer one launch appends the block's L_B sub-block rows and runs its L_B queries over the

@@ -123,6 +123,16 @@ def test_block_decode_step_through_host_buffers(bt):
     assert run.status.item() == 0 and (run.cache.len == w.ctx_blocks).all()
     assert torch.equal(run.out, want_out) and torch.equal(run.cache.k, want_k)
     assert torch.equal(run._host["out"], want_out.cpu())   # and the host copy of the result
+    # the same step as one CUDA-graph replay (copies included), as bench.py times it
+    run.capture_host()
+    run.cache.k[:, :, :, w.ctx_blocks - 1].zero_()
+    run.out.zero_()
+    run._host["out"].zero_()
+    run.replay_host()
+    torch.cuda.synchronize()
+    assert run.status.item() == 0 and (run.cache.len == w.ctx_blocks).all()
+    assert torch.equal(run.out, want_out) and torch.equal(run.cache.k, want_k)
+    assert torch.equal(run._host["out"], want_out.cpu())
 
 
 def test_token_decode_full_size_two_blocks(bt):
