@@ -43,6 +43,10 @@ def test_split_choice_and_workspace(bt):
     assert s > 1 and bt.bt_workspace_bytes(tiny) == s * 4 * 8 * 68 * 4 + counters(4, 8)
     forced = bt.make_config(4, 8, 64, 4, 1, 64, 2, decode_splits=7)
     assert bt.bt_decode_splits(forced) == 7
+    # the choice aims at about 512 work items of at least 128 rows (short caches: up to 4 parts of >= 16 rows)
+    for (B, H, N), want in {(1, 16, 8192): 32, (1, 16, 2048): 16, (8, 16, 8192): 4, (16, 16, 4096): 2,
+                            (64, 16, 4096): 1, (4, 8, 64): 4, (2, 2, 20): 1}.items():
+        assert bt.bt_decode_splits(bt.make_config(B, H, 64, 4, 1, N, 1)) == want, (B, H, N)
     bad = bt.make_config(4, 8, 48, 4, 1, 64, 2)
     assert bt.bt_decode_splits(bad) == 0 and bt.bt_workspace_bytes(bad) == 0
 
