@@ -2,7 +2,7 @@
 // is bound by how many bytes of K and V it keeps in flight, so the bytes are moved by the bulk-copy
 // engine into shared-memory rings and the warps only compute.
 //
-// One persistent CTA per SM, eight warps.  Every warp works alone: it owns a ring of three 8 KB
+// One persistent CTA per SM, six to nine warps (picked per launch).  Every warp works alone: it owns a ring of three 8 KB
 // stages (one stage = a chunk of K rows and the same rows of V), takes whole work items
 // ((sequence, head) or (sequence, head, split)), and lane 0 keeps two chunks in flight with
 // cp.async.bulk while the warp consumes the third - across item boundaries, so the stream never
