@@ -2,11 +2,11 @@
 // is bound by how many bytes of K and V it keeps in flight, so the bytes are moved by the bulk-copy
 // engine into shared-memory rings and the warps only compute.
 //
-// One persistent CTA per SM, six to nine warps (picked per launch).  Every warp works alone: it owns a ring of three 8 KB
-// stages (one stage = a chunk of K rows and the same rows of V), takes whole work items
-// ((sequence, head) or (sequence, head, split)), and lane 0 keeps two chunks in flight with
-// cp.async.bulk while the warp consumes the third - across item boundaries, so the stream never
-// drains.  No CTA-wide synchronisation exists; a stage is handed back by __syncwarp.  Per chunk a
+// One persistent CTA per SM, six to nine warps (picked per launch).  Every warp works alone: it owns
+// a ring of two or three 8 KB stages (depth picked per launch; one stage = a chunk of K rows and the
+// same rows of V), takes whole work items ((sequence, head) or (sequence, head, split)), and lane 0
+// re-requests a stage with cp.async.bulk as soon as its rows are in registers - across item
+// boundaries, so the stream never drains.  No CTA-wide synchronisation exists; a stage is handed back by __syncwarp.  Per chunk a
 // lane group of hd/8 lanes owns a row: 128-bit shared-memory reads, fp32 dot product reduced by
 // shuffles, online softmax in the log2 domain per lane; row groups merge by shuffles at the end of
 // the item.  Every wait on a copy is bounded and raises BT_DEV_TIMEOUT when it runs out.
@@ -42,7 +42,11 @@ namespace ring {
 constexpr int kWarps = BT_DEC_WARPS;
 constexpr int kMinWarps = 6, kMaxWarps = BT_DEC_MAX_WARPS;
 constexpr int kMaxThreads = kMaxWarps * 32;
-constexpr int kStages = BT_DEC_STAGES;
+// Ring depth, chosen per launch: two stages when at least three warps in four have an item (with the
+// memory system saturated by many rings, less in flight per warp runs faster: 82.4 vs 84.2 us at 4096
+// items of 512 rows, 158 vs 164 us at 1024 items of 4096 rows), kDeepStages when only some of the warps
+// have an item and each must cover more of the latency on its own (27.5 vs 28.7 us at 512 items).
+constexpr int kDeepStages = BT_DEC_STAGES;
 constexpr int kUnroll = BT_DEC_UNROLL;     // rows per lane group per chunk
 constexpr int kPrefetchChunks = 16;         // chunks of a warp's first item warmed in L2 ahead of the dependent-launch wait
 constexpr uint32_t kPollLimit = 1u << 24;  // polls of one wait before giving up (each poll suspends briefly)
@@ -56,7 +60,7 @@ struct Geo {
     static constexpr int STAGE_BYTES = 2 * CHUNK_BYTES;   // K chunk, then V chunk
 };
 template <int HD>
-constexpr int smem_bytes(int warps) { return warps * kStages * Geo<HD>::STAGE_BYTES + warps * kStages * 8; }
+constexpr int smem_bytes(int warps, int stages) { return warps * stages * Geo<HD>::STAGE_BYTES + warps * stages * 8; }
 
 __device__ __forceinline__ bool mbar_wait_bounded(uint32_t bar, uint32_t parity) { return mbar_wait_polls(bar, parity, kPollLimit); }
 // bytes global -> shared, completion counted on the mbarrier; the rows are read once, so they are
@@ -107,7 +111,7 @@ __device__ __forceinline__ Work decode_work(int item, const DecodeArgs& a)
 // output directly; otherwise each item writes its normalised partial (hd floats, then its
 // log2-sum-exp; hd+4 floats apart so that every partial is 16-byte aligned) to the workspace and the
 // last one to arrive combines them.
-template <int HD>
+template <int HD, int kStages>
 __global__ void __launch_bounds__(kMaxThreads, 1) block_decode_ring_kernel(DecodeArgs a)
 {
     using G = Geo<HD>;
@@ -375,18 +379,29 @@ __global__ void __launch_bounds__(kMaxThreads, 1) block_decode_ring_kernel(Decod
     }
 }
 
+template <int HD, int STAGES>
+static cudaError_t launch_st(const DecodeArgs& a, long long grid, int warps, bool first_on_device, cudaStream_t stream)
+{
+    if (first_on_device) {
+        cudaError_t e = cudaFuncSetAttribute(block_decode_ring_kernel<HD, STAGES>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                             smem_bytes<HD>(kMaxWarps, STAGES));
+        if (e != cudaSuccess) return e;
+    }
+    return launch_pdl(block_decode_ring_kernel<HD, STAGES>, dim3((unsigned)grid), dim3(warps * 32),
+                      (size_t)smem_bytes<HD>(warps, STAGES), stream, a);
+}
+
 template <int HD>
 static cudaError_t launch_t(const DecodeArgs& a, cudaStream_t stream)
 {
     constexpr int kMaxDevices = 64;
-    static int sm_count[kMaxDevices];  // 0 = this device has not been set up yet
+    static int sm_count[kMaxDevices];   // 0 = this device has not been set up yet
+    static bool ready[kMaxDevices][2];  // per ring depth: the kernel's shared-memory limit is raised
     int dev = 0;
     cudaError_t e = cudaGetDevice(&dev);
     if (e != cudaSuccess) return e;
     if (dev < 0 || dev >= kMaxDevices) return cudaErrorInvalidDevice;
     if (!sm_count[dev]) {
-        e = cudaFuncSetAttribute(block_decode_ring_kernel<HD>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem_bytes<HD>(kMaxWarps));
-        if (e != cudaSuccess) return e;
         int n = 0;
         e = cudaDeviceGetAttribute(&n, cudaDevAttrMultiProcessorCount, dev);
         if (e != cudaSuccess) return e;
@@ -409,7 +424,11 @@ static cudaError_t launch_t(const DecodeArgs& a, cudaStream_t stream)
             warps = w;
         }
     }
-    return launch_pdl(block_decode_ring_kernel<HD>, dim3((unsigned)grid), dim3(warps * 32), (size_t)smem_bytes<HD>(warps), stream, a);
+    const bool shallow = items * 4 >= grid * warps * 3;   // (nearly) every warp has an item: the shallow ring
+    const bool first = !ready[dev][shallow];
+    e = shallow ? launch_st<HD, 2>(a, grid, warps, first, stream) : launch_st<HD, kDeepStages>(a, grid, warps, first, stream);
+    if (e == cudaSuccess) ready[dev][shallow] = true;
+    return e;
 }
 
 }  // namespace ring
