@@ -32,8 +32,8 @@ FALLBACK_PEAKS = {"hbm_gbs": 6650.0, "bf16_tflops": 1590.0, "bf16_tflops_sustain
 # DRAM traffic per launch of the dominant kernel, from the ncu captures summarised under profiles/
 # (dram__bytes_read.sum + dram__bytes_write.sum); None until a capture exists.
 NCU_TRAFFIC_BYTES = {
-    # profiles/block_decode_ring_kernel_config2.md: 274.4 MB on the B=128 capture, traffic is proportional to B
-    "block_decode": 548.8e6,
+    # profiles/block_decode_ring_kernel_config2.md: 274.2 MB on the B=128 capture, traffic is proportional to B
+    "block_decode": 548.4e6,
     # profiles/block_decode_mq_kernel_dense_decode.md: 274.5 MB on the B=32 capture, traffic is proportional to B
     "dense_decode": 2196.0e6,
     # profiles/token_step_pipelined_kernel_config3.md: reads equal the algorithmic reads at j = 0 and j = 3 (25.2 + j x 16.8 MB);
