@@ -19,9 +19,14 @@
  *     thought of as [B][H][hd]).
  *   - `stream` is a cudaStream_t passed as void*.  All work is enqueued on it and
  *     the call returns without synchronising.
+ *   - Alignment: the kernels move data in 16-byte pieces, so every tensor pointer
+ *     (q, k_new, v_new, out, the cache bases, the workspace, the staging buffers)
+ *     must be 16-byte aligned and every int32 / uint32 array 4-byte aligned; a
+ *     pointer that is not is refused with BT_ERR_UNSUPPORTED.
  *   - Host-detectable errors (null pointer, bad shape, unsupported head_dim, a
- *     request larger than the capacity, workspace too small) return a non-zero
- *     bt_status before anything is launched.  Data-dependent conditions found on
+ *     misaligned pointer, a request larger than the capacity, workspace too small)
+ *     return a non-zero bt_status before anything is enqueued: no launch, no copy,
+ *     no memset.  Data-dependent conditions found on
  *     the device (a sequence whose cache is full, attention over an empty cache)
  *     never trap: the sequence is skipped or zeros are produced, and a BT_DEV_*
  *     bit is OR-ed into *dev_status (a device uint32 the caller clears and reads
@@ -45,7 +50,7 @@ typedef enum {
     BT_OK = 0,
     BT_ERR_NULL = 1,        /* a required pointer is NULL                         */
     BT_ERR_SHAPE = 2,       /* non-positive or inconsistent dimension, bad layer  */
-    BT_ERR_UNSUPPORTED = 3, /* head_dim not in {64,128}, too many heads, ...      */
+    BT_ERR_UNSUPPORTED = 3, /* head_dim not in {64,128}, too many heads, misaligned pointer */
     BT_ERR_CAPACITY = 4,    /* n_new larger than the cache capacity               */
     BT_ERR_WORKSPACE = 5,   /* workspace NULL or smaller than bt_workspace_bytes  */
     BT_ERR_CUDA = 6         /* a CUDA runtime call or launch failed               */
@@ -176,7 +181,8 @@ bt_status bt_block_decode_step_multi(const bt_config* cfg, bt_block_cache* cache
  * with a latency budget cannot accept).  Neither this call nor anything it reaches allocates or
  * frees device memory.
  *   - Limit: bt_workspace_bytes(cfg) must not exceed BT_STATIC_WORKSPACE_BYTES, else
- *     BT_ERR_WORKSPACE is returned and nothing is launched.  Every GPU on which the library is
+ *     BT_ERR_WORKSPACE is returned.  Like every refused call, one refused here has enqueued
+ *     nothing and has not touched the shared array.  Every GPU on which the library is
  *     loaded holds that many bytes until the process exits.
  *   - The first call on each device whose config splits the row range looks up the array's
  *     address on that device (the device must be current, as for every call here, and own the
@@ -234,8 +240,9 @@ bt_status bt_token_decode_attn(const bt_config* cfg, bt_local_cache* cache, int 
  * q, out: [B][H][T][hd].  k, v: rows hd apart; (b,h) slab s starts s * kv_seq_stride rows
  * after the base, so kv_seq_stride = T for packed tensors and = N_max when k, v point at a
  * layer of a block cache that already holds the prompt's rows.  Requires kv_seq_stride >= T.
- * Runs on the tensor cores (TMA-fed tcgen05 MMA, accumulators in tensor memory) when all four
- * pointers are 16-byte aligned, else on a CUDA-core kernel.  Every wait inside the tensor-core
+ * Runs on the tensor cores (TMA-fed tcgen05 MMA, accumulators in tensor memory), or, when
+ * cfg->prefill_plain is set, on a CUDA-core kernel (an order of magnitude slower; a cross-check).
+ * The library never switches between the two on its own.  Every wait inside the tensor-core
  * kernel is bounded; one that runs out raises BT_DEV_TIMEOUT in *dev_status and leaves the
  * affected output rows unwritten.
  */
@@ -255,6 +262,21 @@ bt_status bt_block_decode_step_host(const bt_config* cfg, bt_block_cache* cache,
                                     void* out_host, void* q_dev, void* k_dev, void* v_dev, void* out_dev,
                                     void* workspace, size_t workspace_bytes, uint32_t* dev_status,
                                     void* stream);
+
+/*
+ * Self-test of the bounded waits (test support; the paper has no counterpart).  Every wait inside the
+ * library's kernels is on a shared-memory barrier and is bounded - by a poll count in the streaming
+ * decode kernels, by wall time in the prefill kernel - and raises BT_DEV_TIMEOUT when the bound runs
+ * out.  This call launches one small CTA that runs those same two wait routines, with short limits
+ * (a few thousand polls; 0.2 ms), on barriers that nothing will ever complete, plus a control wait on
+ * a completed barrier.  No copy is issued, so nothing is in flight when the waits give up; the kernel
+ * ends normally and the context stays usable.
+ *   report     : optional device uint32[4]: [0] the poll-bounded wait gave up (1 expected),
+ *                [1] the time-bounded wait gave up (1 expected), [2] the control wait succeeded
+ *                (1 expected), [3] nanoseconds the time-bounded wait took.
+ *   dev_status : required; BT_DEV_TIMEOUT is OR-ed in when a wait gave up.
+ */
+bt_status bt_selftest_bounded_wait(uint32_t* report, uint32_t* dev_status, void* stream);
 
 #ifdef __cplusplus
 }

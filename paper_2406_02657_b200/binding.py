@@ -21,7 +21,7 @@ EXPORTS = [
     "bt_version", "bt_status_string", "bt_decode_splits", "bt_workspace_bytes", "bt_block_kv_append",
     "bt_block_decode_attn", "bt_local_kv_reset", "bt_local_kv_append", "bt_token_decode_attn",
     "bt_block_prefill_attn", "bt_block_decode_step_host", "bt_block_decode_attn_noalloc",
-    "bt_workspace_init", "bt_block_decode_step", "bt_block_decode_step_multi",
+    "bt_workspace_init", "bt_block_decode_step", "bt_block_decode_step_multi", "bt_selftest_bounded_wait",
 ]
 
 
@@ -72,6 +72,7 @@ def _load() -> ctypes.CDLL:
     lib.bt_block_decode_step_host.argtypes = [cfgp, ctypes.POINTER(bt_block_cache), i32, vp, vp, vp, vp,
                                               vp, vp, vp, vp, vp, u64, vp, vp]
     lib.bt_block_decode_attn_noalloc.argtypes = [cfgp, ctypes.POINTER(bt_block_cache), i32, vp, vp, vp, vp]
+    lib.bt_selftest_bounded_wait.argtypes = [vp, vp, vp]
     for name in EXPORTS[4:]:
         getattr(lib, name).restype = ctypes.c_int
     return lib
@@ -199,6 +200,11 @@ def bt_block_decode_attn_noalloc(cfg, cache: BlockCache, layer, q, out, dev_stat
     BT_STATIC_WORKSPACE_BYTES; calls on one device share the scratch, so do not overlap them."""
     _check(_lib.bt_block_decode_attn_noalloc(ctypes.byref(cfg), ctypes.byref(cache.c), layer, _ptr(q), _ptr(out),
                                              _ptr(dev_status), _stream(stream)), "bt_block_decode_attn_noalloc")
+
+
+def bt_selftest_bounded_wait(report, dev_status, stream=None):
+    """Run the library's two bounded-wait routines on barriers nothing completes (test support)."""
+    _check(_lib.bt_selftest_bounded_wait(_ptr(report), _ptr(dev_status), _stream(stream)), "bt_selftest_bounded_wait")
 
 
 def bt_local_kv_reset(cfg, cache: LocalCache, layer, seq_mask=None, stream=None):

@@ -83,11 +83,46 @@ bt::CacheView local_view(const bt_config* c, const bt_local_cache* cache, int la
 
 inline bt_status cuda_status(cudaError_t e) { return e == cudaSuccess ? BT_OK : BT_ERR_CUDA; }
 
+// The kernels move data in 16-byte pieces (128-bit loads and stores, cp.async, bulk and tensor copies):
+// every tensor base must sit on a 16-byte boundary, length arrays on a 4-byte one.  NULL passes (it
+// is either optional or refused as BT_ERR_NULL elsewhere).
+inline bool al16(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 15u) == 0; }
+inline bool al4(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 3u) == 0; }
+inline bool block_cache_aligned(const bt_block_cache* c) { return al16(c->k) && al16(c->v) && al4(c->len); }
+inline bool local_cache_aligned(const bt_local_cache* c) { return al16(c->kv) && al4(c->len); }
+
+// what bt_block_decode_attn (k_new == NULL) and bt_block_decode_step check before anything is enqueued
+bt_status decode_validate(const bt_config* cfg, const bt_block_cache* cache, int layer, const void* q, const void* k_new,
+                                 const void* v_new, bool step, const void* out, const void* workspace, size_t workspace_bytes,
+                                 const uint32_t* dev_status)
+{
+    bt_status st = check_config(cfg, layer);
+    if (st != BT_OK) return st;
+    if (!cache || !cache->k || !cache->v || !cache->len || !q || !out) return BT_ERR_NULL;
+    if (step && (!k_new || !v_new)) return BT_ERR_NULL;
+    const bool need_ws = choose_splits(cfg) > 1 || step;
+    if (need_ws && (!workspace || workspace_bytes < bt_workspace_bytes(cfg))) return BT_ERR_WORKSPACE;
+    if (!block_cache_aligned(cache) || !al16(q) || !al16(out) || !al16(k_new) || !al16(v_new) || !al4(dev_status) ||
+        (need_ws && !al16(workspace)))
+        return BT_ERR_UNSUPPORTED;
+    return BT_OK;
+}
+
 }  // namespace
+
+namespace bt {
+bt_status validate_decode_attn_args(const bt_config* cfg, const bt_block_cache* cache, int layer, const void* q, const void* out,
+                                    const uint32_t* dev_status)
+{
+    // a workspace that cannot be refused: only the other arguments are judged
+    return decode_validate(cfg, cache, layer, q, nullptr, nullptr, false, out, reinterpret_cast<const void*>(uintptr_t(16)),
+                           ~size_t(0), dev_status);
+}
+}  // namespace bt
 
 extern "C" {
 
-int bt_version(void) { return 100; }
+int bt_version(void) { return 200; }
 
 const char* bt_status_string(bt_status s)
 {
@@ -130,6 +165,7 @@ bt_status bt_workspace_init(const bt_config* cfg, void* workspace, size_t worksp
     if (st != BT_OK) return st;
     if (!workspace) return BT_ERR_NULL;
     if (workspace_bytes < bt_workspace_bytes(cfg)) return BT_ERR_WORKSPACE;
+    if (!al16(workspace)) return BT_ERR_UNSUPPORTED;
     return cuda_status(cudaMemsetAsync((char*)workspace + partial_bytes(cfg), 0, counter_bytes(cfg), (cudaStream_t)stream));
 }
 
@@ -141,18 +177,19 @@ bt_status bt_block_kv_append(const bt_config* cfg, bt_block_cache* cache, int la
     if (!cache || !cache->k || !cache->v || !cache->len || !k_new || !v_new) return BT_ERR_NULL;
     if (n_new <= 0) return BT_ERR_SHAPE;
     if (n_new > cfg->max_blocks) return BT_ERR_CAPACITY;
+    if (!block_cache_aligned(cache) || !al16(k_new) || !al16(v_new) || !al4(dev_status)) return BT_ERR_UNSUPPORTED;
     return cuda_status(bt::launch_kv_append(block_view(cfg, cache, layer), cfg->batch, cfg->heads, cfg->head_dim,
                                             k_new, v_new, n_new, dev_status, (cudaStream_t)stream));
 }
 
-// append (optional) + attention in one launch
+// append (optional) + attention in one launch; the arguments have passed decode_validate
 static bt_status decode_launch(const bt_config* cfg, bt_block_cache* cache, int layer, const void* q, const void* k_new,
                                const void* v_new, void* out, void* workspace, size_t workspace_bytes,
                                uint32_t* dev_status, void* stream)
 {
     const int splits = choose_splits(cfg);
     const bool need_ws = splits > 1 || k_new != nullptr;
-    if (need_ws && (!workspace || workspace_bytes < bt_workspace_bytes(cfg))) return BT_ERR_WORKSPACE;
+    (void)workspace_bytes;
     bt::CacheView v = block_view(cfg, cache, layer);
     bt::DecodeArgs a;
     a.q = q;
@@ -178,9 +215,8 @@ bt_status bt_block_decode_attn(const bt_config* cfg, const bt_block_cache* cache
                                void* out, void* workspace, size_t workspace_bytes, uint32_t* dev_status,
                                void* stream)
 {
-    bt_status st = check_config(cfg, layer);
+    bt_status st = decode_validate(cfg, cache, layer, q, nullptr, nullptr, false, out, workspace, workspace_bytes, dev_status);
     if (st != BT_OK) return st;
-    if (!cache || !cache->k || !cache->v || !cache->len || !q || !out) return BT_ERR_NULL;
     // without a row to append the kernel only reads the cache
     return decode_launch(cfg, const_cast<bt_block_cache*>(cache), layer, q, nullptr, nullptr, out, workspace,
                          workspace_bytes, dev_status, stream);
@@ -190,9 +226,8 @@ bt_status bt_block_decode_step(const bt_config* cfg, bt_block_cache* cache, int 
                                const void* k_new, const void* v_new, void* out, void* workspace,
                                size_t workspace_bytes, uint32_t* dev_status, void* stream)
 {
-    bt_status st = check_config(cfg, layer);
+    bt_status st = decode_validate(cfg, cache, layer, q, k_new, v_new, true, out, workspace, workspace_bytes, dev_status);
     if (st != BT_OK) return st;
-    if (!cache || !cache->k || !cache->v || !cache->len || !q || !k_new || !v_new || !out) return BT_ERR_NULL;
     return decode_launch(cfg, cache, layer, q, k_new, v_new, out, workspace, workspace_bytes, dev_status, stream);
 }
 
@@ -206,6 +241,7 @@ bt_status bt_block_decode_step_multi(const bt_config* cfg, bt_block_cache* cache
     if (n_q <= 0) return BT_ERR_SHAPE;
     if (n_q > cfg->max_blocks) return BT_ERR_CAPACITY;
     if (!workspace || workspace_bytes < bt_workspace_bytes(cfg)) return BT_ERR_WORKSPACE;
+    if (!block_cache_aligned(cache) || !al16(workspace) || !al4(dev_status)) return BT_ERR_UNSUPPORTED;
     bt::CacheView v = block_view(cfg, cache, layer);
     bt::MultiDecodeArgs a;
     a.q = q;
@@ -233,6 +269,7 @@ bt_status bt_local_kv_reset(const bt_config* cfg, bt_local_cache* cache, int lay
     bt_status st = check_config(cfg, layer);
     if (st != BT_OK) return st;
     if (!cache || !cache->len) return BT_ERR_NULL;
+    if (!al4(cache->len)) return BT_ERR_UNSUPPORTED;
     return cuda_status(bt::launch_len_reset(cache->len + (size_t)layer * cfg->batch, cfg->batch, seq_mask,
                                             (cudaStream_t)stream));
 }
@@ -245,6 +282,7 @@ bt_status bt_local_kv_append(const bt_config* cfg, bt_local_cache* cache, int la
     if (!cache || !cache->kv || !cache->len || !k_new || !v_new) return BT_ERR_NULL;
     if (n_new <= 0) return BT_ERR_SHAPE;
     if (n_new > local_cap(cfg)) return BT_ERR_CAPACITY;
+    if (!local_cache_aligned(cache) || !al16(k_new) || !al16(v_new) || !al4(dev_status)) return BT_ERR_UNSUPPORTED;
     return cuda_status(bt::launch_kv_append(local_view(cfg, cache, layer), cfg->batch, cfg->heads, cfg->head_dim,
                                             k_new, v_new, n_new, dev_status, (cudaStream_t)stream));
 }
@@ -260,6 +298,8 @@ bt_status bt_token_decode_attn(const bt_config* cfg, bt_local_cache* cache, int 
     if (n_q <= 0) return BT_ERR_SHAPE;
     if (!k_new && n_q != 1) return BT_ERR_SHAPE;
     if (n_q > local_cap(cfg)) return BT_ERR_CAPACITY;
+    if (!local_cache_aligned(cache) || !al16(q) || !al16(k_new) || !al16(v_new) || !al16(out) || !al4(dev_status))
+        return BT_ERR_UNSUPPORTED;
     bt::TokenArgs a;
     a.kv = (char*)cache->kv + local_layer_elems(cfg) * layer * 2;
     a.len = cache->len + (size_t)layer * cfg->batch;
@@ -286,6 +326,7 @@ bt_status bt_block_prefill_attn(const bt_config* cfg, const void* q, const void*
     if (st != BT_OK) return st;
     if (!q || !k || !v || !out) return BT_ERR_NULL;
     if (n_blocks <= 0 || kv_seq_stride < n_blocks) return BT_ERR_SHAPE;
+    if (!al16(q) || !al16(k) || !al16(v) || !al16(out) || !al4(dev_status)) return BT_ERR_UNSUPPORTED;
     bt::PrefillArgs a;
     a.q = q;
     a.k = k;
@@ -297,9 +338,11 @@ bt_status bt_block_prefill_attn(const bt_config* cfg, const void* q, const void*
     a.T = n_blocks;
     a.kv_seq_stride = kv_seq_stride;
     a.scale_log2 = scale_log2(cfg);
-    if (!cfg->prefill_plain && bt::prefill_tc_supported(a))
-        return cuda_status(bt::launch_block_prefill_tc(a, dev_status, (cudaStream_t)stream));
-    return cuda_status(bt::launch_block_prefill_simple(a, (cudaStream_t)stream));
+    // the kernel is the caller's choice, never a silent switch: the tensor-core one unless the config asks
+    // for the CUDA-core one
+    if (cfg->prefill_plain) return cuda_status(bt::launch_block_prefill_simple(a, (cudaStream_t)stream));
+    if (!bt::prefill_tc_supported(a)) return BT_ERR_UNSUPPORTED;  // no driver entry point for tensor maps
+    return cuda_status(bt::launch_block_prefill_tc(a, dev_status, (cudaStream_t)stream));
 }
 
 bt_status bt_block_decode_step_host(const bt_config* cfg, bt_block_cache* cache, int layer, const void* q_host,
@@ -307,19 +350,28 @@ bt_status bt_block_decode_step_host(const bt_config* cfg, bt_block_cache* cache,
                                     void* k_dev, void* v_dev, void* out_dev, void* workspace,
                                     size_t workspace_bytes, uint32_t* dev_status, void* stream)
 {
+    // everything bt_block_decode_step would refuse is refused here, before the first copy is enqueued
     bt_status st = check_config(cfg, layer);
     if (st != BT_OK) return st;
-    if (!q_host || !k_new_host || !v_new_host || !out_host || !q_dev || !k_dev || !v_dev || !out_dev)
-        return BT_ERR_NULL;
+    if (!q_host || !k_new_host || !v_new_host || !out_host || !q_dev || !k_dev || !v_dev || !out_dev) return BT_ERR_NULL;
+    st = decode_validate(cfg, cache, layer, q_dev, k_dev, v_dev, true, out_dev, workspace, workspace_bytes, dev_status);
+    if (st != BT_OK) return st;
     const size_t bytes = (size_t)cfg->batch * cfg->heads * cfg->head_dim * 2;
     cudaStream_t s = (cudaStream_t)stream;
     if (cudaMemcpyAsync(k_dev, k_new_host, bytes, cudaMemcpyHostToDevice, s) != cudaSuccess) return BT_ERR_CUDA;
     if (cudaMemcpyAsync(v_dev, v_new_host, bytes, cudaMemcpyHostToDevice, s) != cudaSuccess) return BT_ERR_CUDA;
     if (cudaMemcpyAsync(q_dev, q_host, bytes, cudaMemcpyHostToDevice, s) != cudaSuccess) return BT_ERR_CUDA;
-    st = bt_block_decode_step(cfg, cache, layer, q_dev, k_dev, v_dev, out_dev, workspace, workspace_bytes, dev_status, stream);
+    st = decode_launch(cfg, cache, layer, q_dev, k_dev, v_dev, out_dev, workspace, workspace_bytes, dev_status, stream);
     if (st != BT_OK) return st;
     if (cudaMemcpyAsync(out_host, out_dev, bytes, cudaMemcpyDeviceToHost, s) != cudaSuccess) return BT_ERR_CUDA;
     return BT_OK;
+}
+
+bt_status bt_selftest_bounded_wait(uint32_t* report, uint32_t* dev_status, void* stream)
+{
+    if (!dev_status) return BT_ERR_NULL;
+    if (!al4(report) || !al4(dev_status)) return BT_ERR_UNSUPPORTED;
+    return cuda_status(bt::launch_selftest_bounded_wait(report, dev_status, (cudaStream_t)stream));
 }
 
 }  // extern "C"

@@ -21,6 +21,7 @@
 #include <cuda.h>
 
 #include "bt_common.cuh"
+#include "bt_device.h"
 #include "bt_kernels.h"
 #include "bt_mbarrier.cuh"
 #include "bt_tensor_map.h"
@@ -244,7 +245,7 @@ block_decode_mq_kernel(const __grid_constant__ CUtensorMap mapK, const __grid_co
 
         for (int c = 0; c < w.nchunks; ++c) {
             const uint32_t sidx = consumed % kStages;
-            if (!mbar_wait_bounded(bar0 + 8 * sidx, (consumed / kStages) & 1)) {
+            if (!__all_sync(0xffffffffu, mbar_wait_bounded(bar0 + 8 * sidx, (consumed / kStages) & 1))) {  // warp-uniform outcome
                 alive = false;
                 break;
             }
@@ -385,27 +386,19 @@ template <int HD>
 static cudaError_t launch_multi_t(const MultiDecodeArgs& a, cudaStream_t stream)
 {
     using namespace mq;
-    constexpr int kMaxDevices = 64;
-    static int sm_count[kMaxDevices];  // 0 = this device has not been set up yet
-    int dev = 0;
-    cudaError_t e = cudaGetDevice(&dev);
+    static PerDeviceOnce limit_raised;
+    int dev = 0, sms = 0;
+    cudaError_t e = current_device(&dev, &sms);
     if (e != cudaSuccess) return e;
-    if (dev < 0 || dev >= kMaxDevices) return cudaErrorInvalidDevice;
-    if (!sm_count[dev]) {
-        e = cudaFuncSetAttribute(block_decode_mq_kernel<HD>, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemBytes);
-        if (e != cudaSuccess) return e;
-        int n = 0;
-        e = cudaDeviceGetAttribute(&n, cudaDevAttrMultiProcessorCount, dev);
-        if (e != cudaSuccess) return e;
-        sm_count[dev] = n > 0 ? n : 1;
-    }
+    e = raise_smem_limit_once(limit_raised, dev, block_decode_mq_kernel<HD>, kSmemBytes);
+    if (e != cudaSuccess) return e;
     const long long items = (long long)a.B * a.H;
     if (items > 0x7fffffffLL - 4096) return cudaErrorInvalidConfiguration;
     CUtensorMap mk, mv;
     if (!make_slab_map(&mk, a.k, HD, a.n_max, a.n_max, items, Geo<HD>::ROWS) ||
         !make_slab_map(&mv, a.v, HD, a.n_max, a.n_max, items, Geo<HD>::ROWS))
         return cudaErrorInvalidValue;
-    const long long grid = items < sm_count[dev] ? items : sm_count[dev];
+    const long long grid = items < sms ? items : sms;
     return launch_pdl(block_decode_mq_kernel<HD>, dim3((unsigned)grid), dim3(kThreads), (size_t)kSmemBytes, stream, mk, mv, a);
 }
 

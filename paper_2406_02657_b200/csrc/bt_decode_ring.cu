@@ -19,6 +19,7 @@
 // it; the sequence's length is raised by the item that is last to finish with that sequence, once
 // every item has read the old one.  Both counters return to zero before the kernel ends.
 #include "bt_common.cuh"
+#include "bt_device.h"
 #include "bt_kernels.h"
 #include "bt_mbarrier.cuh"
 
@@ -230,7 +231,8 @@ __global__ void __launch_bounds__(kMaxThreads, 1) block_decode_ring_kernel(Decod
         const int nchunks = (w.c1 - w.r0 + ROWS - 1) / ROWS;
         for (int c = 0; c < nchunks; ++c) {
             const uint32_t sidx = consumed % kStages;
-            if (!mbar_wait_bounded(bar0 + 8 * sidx, (consumed / kStages) & 1)) {
+            // the outcome is made warp-uniform: the shuffles and __syncwarp below need all 32 lanes
+            if (!__all_sync(0xffffffffu, mbar_wait_bounded(bar0 + 8 * sidx, (consumed / kStages) & 1))) {
                 alive = false;
                 break;
             }
@@ -380,13 +382,11 @@ __global__ void __launch_bounds__(kMaxThreads, 1) block_decode_ring_kernel(Decod
 }
 
 template <int HD, int STAGES>
-static cudaError_t launch_st(const DecodeArgs& a, long long grid, int warps, bool first_on_device, cudaStream_t stream)
+static cudaError_t launch_st(const DecodeArgs& a, long long grid, int warps, int dev, cudaStream_t stream)
 {
-    if (first_on_device) {
-        cudaError_t e = cudaFuncSetAttribute(block_decode_ring_kernel<HD, STAGES>, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                                             smem_bytes<HD>(kMaxWarps, STAGES));
-        if (e != cudaSuccess) return e;
-    }
+    static PerDeviceOnce limit_raised;
+    cudaError_t e = raise_smem_limit_once(limit_raised, dev, block_decode_ring_kernel<HD, STAGES>, smem_bytes<HD>(kMaxWarps, STAGES));
+    if (e != cudaSuccess) return e;
     return launch_pdl(block_decode_ring_kernel<HD, STAGES>, dim3((unsigned)grid), dim3(warps * 32),
                       (size_t)smem_bytes<HD>(warps, STAGES), stream, a);
 }
@@ -394,23 +394,13 @@ static cudaError_t launch_st(const DecodeArgs& a, long long grid, int warps, boo
 template <int HD>
 static cudaError_t launch_t(const DecodeArgs& a, cudaStream_t stream)
 {
-    constexpr int kMaxDevices = 64;
-    static int sm_count[kMaxDevices];   // 0 = this device has not been set up yet
-    static bool ready[kMaxDevices][2];  // per ring depth: the kernel's shared-memory limit is raised
-    int dev = 0;
-    cudaError_t e = cudaGetDevice(&dev);
+    int dev = 0, sms = 0;
+    cudaError_t e = current_device(&dev, &sms);
     if (e != cudaSuccess) return e;
-    if (dev < 0 || dev >= kMaxDevices) return cudaErrorInvalidDevice;
-    if (!sm_count[dev]) {
-        int n = 0;
-        e = cudaDeviceGetAttribute(&n, cudaDevAttrMultiProcessorCount, dev);
-        if (e != cudaSuccess) return e;
-        sm_count[dev] = n > 0 ? n : 1;
-    }
     const long long items = (long long)a.B * a.H * a.splits;
     if (items > 0x7fffffffLL - 4096) return cudaErrorInvalidConfiguration;
     // one CTA per SM; with few items, one item per CTA first so that they spread over the SMs
-    long long grid = items < sm_count[dev] ? items : sm_count[dev];
+    long long grid = items < sms ? items : sms;
     // Items are dealt whole, so the launch takes ceil(items / warps) rounds and the warps of the last round
     // that have no item idle while a warp cannot stream faster than its ring allows: pick the warp count
     // with the fullest last round (4096 items on 148 SMs: 7 warps run 3.95 -> 4 rounds, 8 warps 3.46 -> 4).
@@ -425,10 +415,7 @@ static cudaError_t launch_t(const DecodeArgs& a, cudaStream_t stream)
         }
     }
     const bool shallow = items * 4 >= grid * warps * 3;   // (nearly) every warp has an item: the shallow ring
-    const bool first = !ready[dev][shallow];
-    e = shallow ? launch_st<HD, 2>(a, grid, warps, first, stream) : launch_st<HD, kDeepStages>(a, grid, warps, first, stream);
-    if (e == cudaSuccess) ready[dev][shallow] = true;
-    return e;
+    return shallow ? launch_st<HD, 2>(a, grid, warps, dev, stream) : launch_st<HD, kDeepStages>(a, grid, warps, dev, stream);
 }
 
 }  // namespace ring

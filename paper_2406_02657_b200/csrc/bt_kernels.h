@@ -5,7 +5,16 @@
 #include <cuda_runtime.h>
 #include <stdint.h>
 
+#include "../../include/bt.h"
+
 namespace bt {
+
+// Everything bt_block_decode_attn checks on the host except the workspace (for the entry point that
+// supplies the workspace itself and must refuse bad arguments before it enqueues anything).
+bt_status validate_decode_attn_args(const bt_config* cfg, const bt_block_cache* cache, int layer, const void* q, const void* out,
+                                    const uint32_t* dev_status);
+// Test-only kernel behind bt_selftest_bounded_wait.
+cudaError_t launch_selftest_bounded_wait(uint32_t* report, uint32_t* dev_status, cudaStream_t stream);
 
 // Rows of a cache as the copy kernels see them: K row r of slab s at
 // k + s*slab_stride + r*row_stride (elements), V likewise from v.

@@ -55,4 +55,33 @@ __device__ __forceinline__ bool mbar_wait_polls(uint32_t bar, uint32_t parity, u
     return false;
 }
 
+
+__device__ __forceinline__ uint64_t global_ns()
+{
+    uint64_t t;
+    asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(t));
+    return t;
+}
+// Wait bounded in wall time (limit_ns; the clock is looked at every 64 polls) and in polls (spin_limit),
+// for kernels whose threads wait on one another: *abort_flag is a shared-memory word that a thread sets
+// when its own wait runs out and that every waiting thread of the CTA watches, so that one failed wait
+// winds the whole CTA down.  Returns false when the limit ran out here or another thread gave up.
+__device__ __forceinline__ bool mbar_wait_walltime(uint32_t bar, uint32_t parity, volatile int* abort_flag, uint32_t spin_limit,
+                                                   uint64_t limit_ns)
+{
+    if (mbar_test_wait(bar, parity)) return true;
+    uint64_t t0 = 0;
+    for (uint32_t it = 0; it < spin_limit; ++it) {
+        if (mbar_try_wait(bar, parity)) return true;
+        if ((it & 63u) == 63u) {
+            if (*abort_flag) return false;
+            const uint64_t now = global_ns();
+            if (t0 == 0) t0 = now;
+            else if (now - t0 > limit_ns) break;
+        }
+    }
+    *abort_flag = 1;
+    return false;
+}
+
 }  // namespace bt

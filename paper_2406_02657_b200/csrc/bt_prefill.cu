@@ -23,6 +23,7 @@
 #include <cuda.h>
 
 #include "bt_common.cuh"
+#include "bt_device.h"
 #include "bt_kernels.h"
 #include "bt_mbarrier.cuh"
 #include "bt_tensor_map.h"
@@ -37,39 +38,11 @@ constexpr uint32_t kSpinLimit = 1u << 26;
 constexpr uint64_t kWaitLimitNs = 1000000000ull;  // 1 s: far beyond any legitimate wait
 constexpr float kRescaleThreshold = 8.0f;  // log2 units
 
-// Optional event timeline (compiled in only with -DBT_PF_TRACE; a development aid, off in the library):
-// CTA 0 records (clock, event id) pairs per role into p.trace[role][kTraceEvents].
-#ifdef BT_PF_TRACE
-constexpr int kTraceEvents = 4096;
-#define PF_EV_DECL int ev_n = 0
-#define PF_EV(role, id) do { if (p.trace && blockIdx.x == 0 && ev_n < kTraceEvents) { p.trace[(role) * kTraceEvents + ev_n] = (clock64() << 8) | (long long)(id); ++ev_n; } } while (0)
-#else
-#define PF_EV_DECL
-#define PF_EV(role, id)
-#endif
-
-__device__ __forceinline__ uint64_t global_ns()
-{
-    uint64_t t;
-    asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(t));
-    return t;
-}
 // Bounded wait: gives up after kWaitLimitNs of wall time (or kSpinLimit polls).  Returns false when
-// the limit ran out or another thread of the CTA gave up.
+// the limit ran out (BT_DEV_TIMEOUT is raised) or another thread of the CTA gave up.
 __device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatile int* abort_flag, uint32_t* dev_status)
 {
-    if (mbar_test_wait(bar, parity)) return true;
-    uint64_t t0 = 0;
-    for (uint32_t it = 0; it < kSpinLimit; ++it) {
-        if (mbar_try_wait(bar, parity)) return true;
-        if ((it & 63u) == 63u) {
-            if (*abort_flag) return false;
-            const uint64_t now = global_ns();
-            if (t0 == 0) t0 = now;
-            else if (now - t0 > kWaitLimitNs) break;
-        }
-    }
-    *abort_flag = 1;
+    if (mbar_wait_walltime(bar, parity, abort_flag, kSpinLimit, kWaitLimitNs)) return true;
     raise_status(dev_status, BT_DEV_TIMEOUT);
     return false;
 }
@@ -271,13 +244,7 @@ struct Params {
     int T, n_qtiles, n_classes;
     long long n_items;
     float scale_log2;
-#ifdef BT_PF_TRACE
-    long long* trace;
-#endif
 };
-#ifdef BT_PF_TRACE
-long long* g_trace = nullptr;
-#endif
 
 // warps 0-3: softmax warpgroup of tile A, warps 4-7: of tile B
 constexpr int kProducerWarp = 8, kMmaWarp = 9;
@@ -442,24 +409,19 @@ block_prefill_tc_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_c
             uint32_t p_count[2] = {0, 0};         // P tiles consumed so far, per query tile slot
             bool ok = true;
             uint32_t n_done = 0;
-            PF_EV_DECL;
             for (long long item = blockIdx.x; ok && item < p.n_items; item += gridDim.x, ++n_done) {
                 const Item it = decode_item(item, p);
-                PF_EV(2, 20);
                 const int qbuf[2] = {(n_done & 1) ? 2 : 0, 1};
                 const int steps[2] = {it.na, it.nb};
                 // S_x(j) = Q_x K_j^T, then the barriers that fire when it (and all before it) is done
                 auto issue_s = [&](int x, int j) {
                     const uint32_t kc = kv_base + j, st = kc % kKvStages;
-                    PF_EV(2, 0 + 32 * x);
                     ok = ok && mbar_wait(bar(B_KFULL + st), (kc / kKvStages) & 1, abort_flag, p.dev_status);
-                    PF_EV(2, 1 + 32 * x);
                     if (ok && j == 0) {
                         ok = mbar_wait(bar(B_QFULL + qbuf[x]), q_uses[qbuf[x]] & 1, abort_flag, p.dev_status);
                         ++q_uses[qbuf[x]];
                     }
                     if (!ok) return;
-                    PF_EV(2, 2 + 32 * x);
                     tc_fence_after();
                     const uint32_t q0 = sQ + qbuf[x] * TILE_BYTES, k0 = sK + st * TILE_BYTES;
 #pragma unroll
@@ -472,15 +434,12 @@ block_prefill_tc_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_c
                     if (j == steps[x] - 1) mma_commit(bar(B_QEMPTY + qbuf[x]));  // last use of this Q tile
                     // K_j is free after its last reader: tile B while it still runs, else tile A
                     if (x == 1 || j >= it.nb) mma_commit(bar(B_KEMPTY + st));
-                    PF_EV(2, 3 + 32 * x);
                 };
                 // O_x (+)= P_x(j) V_j
                 auto issue_pv = [&](int x, int j) {
                     const uint32_t kc = kv_base + j, st = kc % kKvStages;
                     ok = ok && mbar_wait(bar(B_P0FULL + x), p_count[x] & 1, abort_flag, p.dev_status);
-                    PF_EV(2, 4 + 32 * x);
                     // V_j has landed: a softmax thread waited for it before the last arrival on P0FULL
-                    PF_EV(2, 5 + 32 * x);
                     if (!ok) return;
                     tc_fence_after();
                     const uint32_t v0 = sV + st * TILE_BYTES;
@@ -494,9 +453,7 @@ block_prefill_tc_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_c
                     // the softmax warps still work on the last quarter
 #pragma unroll
                     for (int kk = 0; kk < kEarlyChunks * 2; ++kk) pv(kk);
-                    PF_EV(2, 6 + 32 * x);
                     ok = mbar_wait(bar(B_P1FULL + x), p_count[x] & 1, abort_flag, p.dev_status);
-                    PF_EV(2, 7 + 32 * x);
                     if (!ok) return;
                     ++p_count[x];
                     tc_fence_after();
@@ -507,7 +464,6 @@ block_prefill_tc_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_c
                     // released by the epilogue
                     if ((x == 1 || j >= it.nb) && j != steps[x] - 1) mma_commit(bar(B_VEMPTY + st));
                     if (j == steps[x] - 1) mma_commit(bar(B_OFULL + x));
-                    PF_EV(2, 8 + 32 * x);
                 };
                 issue_s(0, 0);
                 if (it.nb > 0) issue_s(1, 0);
@@ -533,12 +489,6 @@ block_prefill_tc_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_c
         uint32_t s_count = 0, o_count = 0;                 // S tiles / O tiles consumed so far by this thread
         uint32_t kv_base = 0;                              // key/value tiles consumed by earlier items
         bool ok = true;
-        PF_EV_DECL;
-#ifdef BT_PF_TRACE
-#define PF_EVS(id) do { if (wq == 0 && lane == 0) PF_EV(x, id); } while (0)
-#else
-#define PF_EVS(id)
-#endif
         for (long long item = blockIdx.x; ok && item < p.n_items; item += gridDim.x) {
             const Item it = decode_item(item, p);
             const int qt = x ? it.qb : it.qa, n_kv = x ? it.nb : it.na;
@@ -551,7 +501,6 @@ block_prefill_tc_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_c
                 const bool diag = (j == qt);
                 ok = mbar_wait(bar(B_SFULL + x), s_count & 1, abort_flag, p.dev_status);  // S_j ready; O settled
                 if (!ok) break;
-                PF_EVS(1);
                 tc_fence_after();
                 // On the diagonal tile the rows of warp w (32w .. 32w+31) see nothing right of column
                 // 32w+31: only column chunks 0..w are loaded and exponentiated, chunk w with a per-row mask.
@@ -564,7 +513,6 @@ block_prefill_tc_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_c
 #pragma unroll
                 for (int c = 0; c < BN / 32; ++c)
                     if (c < nch) tmem_ld_fence32(sr + c * 32);
-                PF_EVS(2);
                 if (diag) {  // masked scores become -inf: they drop out of the maximum and exponentiate to 0
 #pragma unroll
                     for (int c = 0; c < BN / 32; ++c)
@@ -587,7 +535,6 @@ block_prefill_tc_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_c
                     }
                 float mx = fmaxf(fmaxf(mx4[0], mx4[1]), fmaxf(mx4[2], mx4[3]));
                 mx *= p.scale_log2;
-                PF_EVS(3);
                 float factor = 1.f;
                 const bool grow_ref = mx > m_ref + kRescaleThreshold;  // first tile: m_ref = -inf
                 if (grow_ref) {
@@ -654,7 +601,6 @@ block_prefill_tc_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_c
                             ok = mbar_wait(bar(B_VFULL + kc % kKvStages), (kc / kKvStages) & 1, abort_flag, p.dev_status);
                         }
                         mbar_arrive(bar(B_P0FULL + x));
-                        PF_EVS(4);
                     }
                 }
                 {
@@ -666,14 +612,12 @@ block_prefill_tc_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_c
                 tmem_wait_st();
                 tc_fence_before();
                 mbar_arrive(bar(B_P1FULL + x));
-                PF_EVS(5);
             }
             // From here to the named barrier below no thread leaves early: a thread whose wait ran out (ok ==
             // false; later waits then give up soon, the abort flag being up) still stages its row and meets the others, and the
             // barrier tells all 128 whether any of them failed, so that they give up at the same item.
             if (ok) ok = mbar_wait(bar(B_OFULL + x), o_count & 1, abort_flag, p.dev_status);
             ++o_count;
-            PF_EVS(6);
             tc_fence_after();
             const float inv = l > 0.f ? 1.f / l : 0.f;
             // O row -> bf16 -> the shared-memory stage that held this tile's last V tile (every MMA that
@@ -700,7 +644,6 @@ block_prefill_tc_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_c
             }
             tc_fence_before();
             asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
-            PF_EVS(7);
             uint32_t any_failed;  // the warpgroup's 128 rows are staged; did a wait run out in any of its threads?
             asm volatile(
                 "{\n\t.reg .pred p, q;\n\t"
@@ -718,7 +661,6 @@ block_prefill_tc_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_c
                 asm volatile("cp.async.bulk.wait_group.read 0;" ::: "memory");
                 mbar_arrive(bar(B_VEMPTY + stage_o));
             }
-            PF_EVS(8);
             // the next item's first P V overwrites O: it is issued only after this thread's next
             // arrival on P0FULL, which follows these loads in program order
         }
@@ -754,20 +696,12 @@ static int gcd_int(int a, int b)
 template <int HD>
 static cudaError_t launch_t(const PrefillArgs& a, uint32_t* dev_status, cudaStream_t stream)
 {
-    constexpr int kMaxDevices = 64;
-    static int sm_count[kMaxDevices];  // 0 = this device has not been set up yet
-    int dev = 0;
-    cudaError_t e = cudaGetDevice(&dev);
+    static PerDeviceOnce limit_raised;
+    int dev = 0, sms = 0;
+    cudaError_t e = current_device(&dev, &sms);
     if (e != cudaSuccess) return e;
-    if (dev < 0 || dev >= kMaxDevices) return cudaErrorInvalidDevice;
-    if (!sm_count[dev]) {
-        e = cudaFuncSetAttribute(block_prefill_tc_kernel<HD>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem_bytes<HD>());
-        if (e != cudaSuccess) return e;
-        int n = 0;
-        e = cudaDeviceGetAttribute(&n, cudaDevAttrMultiProcessorCount, dev);
-        if (e != cudaSuccess) return e;
-        sm_count[dev] = n > 0 ? n : 1;
-    }
+    e = raise_smem_limit_once(limit_raised, dev, block_prefill_tc_kernel<HD>, smem_bytes<HD>());
+    if (e != cudaSuccess) return e;
     const long long slabs = (long long)a.B * a.H;
     CUtensorMap mq, mk, mv, mo;
     if (!make_map(&mq, a.q, HD, a.T, a.T, slabs) || !make_map(&mk, a.k, HD, a.T, a.kv_seq_stride, slabs) ||
@@ -780,12 +714,9 @@ static cudaError_t launch_t(const PrefillArgs& a, uint32_t* dev_status, cudaStre
     p.n_classes = (p.n_qtiles + 1) / 2;
     p.n_items = slabs * p.n_classes;
     p.scale_log2 = a.scale_log2;
-#ifdef BT_PF_TRACE
-    p.trace = g_trace;
-#endif
     // one persistent CTA per SM; a grid size coprime to the number of classes makes every CTA
     // cycle through all classes (heavy and light items alike)
-    long long grid = p.n_items < sm_count[dev] ? p.n_items : sm_count[dev];
+    long long grid = p.n_items < sms ? p.n_items : sms;
     while (grid > 1 && p.n_items > grid && gcd_int((int)grid, p.n_classes) != 1) --grid;
     return launch_pdl(block_prefill_tc_kernel<HD>, dim3((unsigned)grid), dim3(kThreads), (size_t)smem_bytes<HD>(), stream, mq, mk, mv, mo, p);
 }

@@ -15,6 +15,7 @@
 #include <mutex>
 
 #include "../../include/bt.h"
+#include "bt_kernels.h"
 
 namespace {
 
@@ -33,7 +34,10 @@ bt_status static_ws_on_current_device(void** addr)
     std::lock_guard<std::mutex> lock(g_ws_mutex);
     if (!g_ws_addr[dev]) {
         void* p = nullptr;
-        if (cudaGetSymbolAddress(&p, g_static_ws) != cudaSuccess || !p) return BT_ERR_CUDA;
+        if (cudaGetSymbolAddress(&p, g_static_ws) != cudaSuccess || !p) {
+            (void)cudaGetLastError();  // the failure is reported here; it must not surface in a later call's launch check
+            return BT_ERR_CUDA;
+        }
         g_ws_addr[dev] = p;
     }
     *addr = g_ws_addr[dev];
@@ -45,12 +49,14 @@ bt_status static_ws_on_current_device(void** addr)
 extern "C" bt_status bt_block_decode_attn_noalloc(const bt_config* cfg, const bt_block_cache* cache, int layer,
                                                   const void* q, void* out, uint32_t* dev_status, void* stream)
 {
-    // 0 for an invalid config too: bt_block_decode_attn below then reports what is wrong with it
-    const size_t need = bt_workspace_bytes(cfg);
-    if (need > (size_t)BT_STATIC_WORKSPACE_BYTES) return BT_ERR_WORKSPACE;
+    // every argument is judged first: a call that is refused has enqueued nothing and has not touched the
+    // shared scratch, which a call already in flight may be using
+    bt_status st = bt::validate_decode_attn_args(cfg, cache, layer, q, out, dev_status);
+    if (st != BT_OK) return st;
+    if (bt_workspace_bytes(cfg) > (size_t)BT_STATIC_WORKSPACE_BYTES) return BT_ERR_WORKSPACE;
     void* ws = nullptr;
-    if (need && bt_decode_splits(cfg) > 1) {
-        bt_status st = static_ws_on_current_device(&ws);
+    if (bt_decode_splits(cfg) > 1) {
+        st = static_ws_on_current_device(&ws);
         if (st != BT_OK) return st;
         // configs of different shapes share the array, and one config's partial results may lie where
         // another's arrival counters do: the counters are zeroed (a memset node, no allocation) every time

@@ -5,6 +5,7 @@
 // loads, a few shuffles and one 128-bit store per tensor.  A CTA always covers whole sequences
 // so that every head reads the old length before one thread writes the new one.
 #include "bt_common.cuh"
+#include "bt_device.h"
 #include "bt_kernels.h"
 
 namespace bt {
@@ -417,17 +418,6 @@ token_step_pipelined_kernel(TokenArgs a, int seqs_per_cta, int threads_per_seq)
     cp_async_wait<0>();
 }
 
-static int sm_count()
-{
-    static int n = 0;
-    if (n == 0) {
-        int dev = 0;
-        if (cudaGetDevice(&dev) != cudaSuccess || cudaDeviceGetAttribute(&n, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess || n <= 0)
-            n = 148;
-    }
-    return n;
-}
-
 #ifndef BT_TOK_DEPTH4
 #define BT_TOK_DEPTH4 1
 #endif
@@ -440,15 +430,14 @@ static cudaError_t launch_pipelined(const TokenArgs& a, int spc, int tps, cudaSt
 {
     constexpr size_t smem = (size_t)(kDepth + 1) * (3 + 2 * kMaxRows) * kTokThreads * sizeof(uint4);
     static_assert(smem * kCtasPerSm <= 224 * 1024, "slots do not fit in shared memory");
-    static bool attr_set = false;
-    if (!attr_set) {
-        cudaError_t e = cudaFuncSetAttribute(token_step_pipelined_kernel<HD, kDepth, kMaxRows, kCtasPerSm>,
-                                             cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
-        if (e != cudaSuccess) return e;
-        attr_set = true;
-    }
+    static PerDeviceOnce limit_raised;
+    int dev = 0, sms = 0;
+    cudaError_t e = current_device(&dev, &sms);
+    if (e != cudaSuccess) return e;
+    e = raise_smem_limit_once(limit_raised, dev, token_step_pipelined_kernel<HD, kDepth, kMaxRows, kCtasPerSm>, (int)smem);
+    if (e != cudaSuccess) return e;
     const int n_groups = (a.B + spc - 1) / spc;
-    const int slots = sm_count() * kCtasPerSm;
+    const int slots = sms * kCtasPerSm;
     const int grid = n_groups < slots ? n_groups : slots;
     return launch_pdl(token_step_pipelined_kernel<HD, kDepth, kMaxRows, kCtasPerSm>, dim3(grid), dim3(kTokThreads), smem, stream,
                       a, spc, tps);

@@ -100,6 +100,73 @@ def test_host_detectable_errors_return_before_launch(bt):
                                        None, 0, None, None) == bt.BT_ERR_NULL
 
 
+def test_misaligned_pointers_are_refused_before_launch(bt):
+    """The kernels use 16-byte loads, stores and copies: a pointer off a 16-byte boundary (a 2-byte-aligned
+    bf16 view, say) would fault on the device, so every entry point refuses it on the host.  Fake
+    addresses: nothing is launched, nothing is dereferenced."""
+    L = bt.lib()
+    ref = ctypes.byref
+    ok, odd, odd4 = ctypes.c_void_p(0x1000), ctypes.c_void_p(0x1002), ctypes.c_void_p(0x1008)
+    cfg = bt.make_config(4, 8, 64, 4, 1, 64, 2, decode_splits=1)
+    split = bt.make_config(4, 8, 64, 4, 1, 64, 2, decode_splits=2)
+    bc = bt.binding.bt_block_cache(0x1000, 0x1000, 0x1000)
+    lc = bt.binding.bt_local_cache(0x1000, 0x1000)
+    U = bt.BT_ERR_UNSUPPORTED
+    big = 1 << 20
+    for bad in (odd, odd4):
+        assert L.bt_block_kv_append(ref(cfg), ref(bc), 0, bad, ok, 1, None, None) == U
+        assert L.bt_block_kv_append(ref(cfg), ref(bc), 0, ok, bad, 1, None, None) == U
+        assert L.bt_block_decode_attn(ref(cfg), ref(bc), 0, bad, ok, None, 0, None, None) == U
+        assert L.bt_block_decode_attn(ref(cfg), ref(bc), 0, ok, bad, None, 0, None, None) == U
+        assert L.bt_block_decode_attn(ref(split), ref(bc), 0, ok, ok, bad, big, None, None) == U
+        assert L.bt_block_decode_attn_noalloc(ref(cfg), ref(bc), 0, bad, ok, None, None) == U
+        assert L.bt_block_decode_step(ref(cfg), ref(bc), 0, ok, bad, ok, ok, ok, big, None, None) == U
+        assert L.bt_block_decode_step(ref(cfg), ref(bc), 0, ok, ok, ok, ok, bad, big, None, None) == U
+        assert L.bt_block_decode_step_multi(ref(cfg), ref(bc), 0, ok, ok, bad, 2, ok, ok, big, None, None) == U
+        assert L.bt_block_decode_step_host(ref(cfg), ref(bc), 0, ok, ok, ok, ok, ok, bad, ok, ok, ok, big, None, None) == U
+        assert L.bt_local_kv_append(ref(cfg), ref(lc), 0, bad, ok, 1, None, None) == U
+        assert L.bt_token_decode_attn(ref(cfg), ref(lc), 0, bad, ok, ok, 1, 0, None, ok, None, None) == U
+        assert L.bt_token_decode_attn(ref(cfg), ref(lc), 0, ok, ok, ok, 1, 0, None, bad, None, None) == U
+        assert L.bt_block_prefill_attn(ref(cfg), ok, bad, ok, 8, 8, ok, None, None) == U
+        assert L.bt_workspace_init(ref(cfg), bad, big, None) == U
+    for k, v, ln in ((0x1002, 0x1000, 0x1000), (0x1000, 0x1008, 0x1000), (0x1000, 0x1000, 0x1002)):
+        mis = bt.binding.bt_block_cache(k, v, ln)
+        assert L.bt_block_decode_attn(ref(cfg), ref(mis), 0, ok, ok, None, 0, None, None) == U
+        assert L.bt_block_kv_append(ref(cfg), ref(mis), 0, ok, ok, 1, None, None) == U
+    for kv, ln in ((0x1004, 0x1000), (0x1000, 0x1001)):
+        mis = bt.binding.bt_local_cache(kv, ln)
+        assert L.bt_token_decode_attn(ref(cfg), ref(mis), 0, ok, ok, ok, 1, 0, None, ok, None, None) == U
+    assert L.bt_local_kv_reset(ref(cfg), ref(bt.binding.bt_local_cache(0x1000, 0x1002)), 0, None, None) == U
+    # a misaligned status word (uint32) is refused too
+    assert L.bt_block_decode_attn(ref(cfg), ref(bc), 0, ok, ok, None, 0, ctypes.c_void_p(0x1002), None) == U
+    # the prefill never changes kernels on its own: the CUDA-core kernel must be asked for, and wants aligned pointers too
+    plain = bt.make_config(4, 8, 64, 4, 1, 64, 2, prefill_plain=1)
+    assert L.bt_block_prefill_attn(ref(plain), ok, odd, ok, 8, 8, ok, None, None) == U
+
+
+def test_refused_calls_enqueue_nothing(bt):
+    """The two entry points that enqueue something before their kernel (host copies; the memset of the
+    shared scratch) judge every argument first: a NULL cache comes back as BT_ERR_NULL although the
+    copy sources / the scratch would have been usable."""
+    L = bt.lib()
+    ref = ctypes.byref
+    ok = ctypes.c_void_p(0x1000)
+    cfg = bt.make_config(4, 8, 64, 4, 1, 64, 2)
+    assert bt.bt_decode_splits(cfg) > 1
+    for k, v, ln in ((0, 0x1000, 0x1000), (0x1000, 0, 0x1000), (0x1000, 0x1000, 0)):
+        nullc = bt.binding.bt_block_cache(k, v, ln)
+        assert L.bt_block_decode_step_host(ref(cfg), ref(nullc), 0, ok, ok, ok, ok, ok, ok, ok, ok, ok, 1 << 20, None, None) \
+            == bt.BT_ERR_NULL
+        assert L.bt_block_decode_attn_noalloc(ref(cfg), ref(nullc), 0, ok, ok, None, None) == bt.BT_ERR_NULL
+    bc = bt.binding.bt_block_cache(0x1000, 0x1000, 0x1000)
+    assert L.bt_block_decode_step_host(ref(cfg), None, 0, ok, ok, ok, ok, ok, ok, ok, ok, ok, 1 << 20, None, None) == bt.BT_ERR_NULL
+    assert L.bt_block_decode_step_host(ref(cfg), ref(bc), 0, ok, ok, ok, ok, ok, ok, ok, ok, None, 0, None, None) == bt.BT_ERR_WORKSPACE
+    assert L.bt_block_decode_step_host(ref(cfg), ref(bc), 5, ok, ok, ok, ok, ok, ok, ok, ok, ok, 1 << 20, None, None) == bt.BT_ERR_SHAPE
+    assert L.bt_block_decode_attn_noalloc(ref(cfg), ref(bc), 0, None, ok, None, None) == bt.BT_ERR_NULL
+    assert L.bt_block_decode_attn_noalloc(ref(cfg), ref(bc), 7, ok, ok, None, None) == bt.BT_ERR_SHAPE
+    assert L.bt_selftest_bounded_wait(None, None, None) == bt.BT_ERR_NULL
+
+
 def test_oracle_is_not_imported_by_the_product():
     pkg = os.path.join(ROOT, "paper_2406_02657_b200")
     for dirpath, _, files in os.walk(pkg):

@@ -204,3 +204,19 @@ def test_block_prefill_full_size(bt):
         q, k, v = (gen.torch_to_bits(x[l, b:b + 1, h:h + 1]) for x in (run.q, run.k, run.v))
         ref = oracle.block_prefill_attn(q, k, v)
         assert_close(run.out[l, b:b + 1, h:h + 1], ref, f"full-size prefill layer {l} b {b} h {h}", p_bf16=True)
+
+
+def test_block_prefill_8k_prompt_full_size(bt):
+    """The 8K-prompt case (2048 prompt blocks, batch 8, 16 heads, head_dim 128), two of the 12 layers:
+    every row written, sampled (sequence, head) pairs against the oracle."""
+    from paper_2406_02657_b200 import harness
+    w = configs.scaled(configs.BLOCK_PREFILL_8K, n_layers=2)
+    run = harness.PrefillRun(w, fill=_fill(w))
+    run.out.fill_(float("nan"))
+    run.step()
+    torch.cuda.synchronize()
+    assert torch.isfinite(run.out.float()).all()
+    for l, b, h in ((0, 0, 0), (0, 7, 15), (1, 3, 8), (1, 7, 0)):
+        q, k, v = (gen.torch_to_bits(x[l, b:b + 1, h:h + 1]) for x in (run.q, run.k, run.v))
+        ref = oracle.block_prefill_attn(q, k, v)
+        assert_close(run.out[l, b:b + 1, h:h + 1], ref, f"8K-prompt prefill layer {l} b {b} h {h}", p_bf16=True)

@@ -86,7 +86,13 @@ def test_tiny_prefill_packed_and_from_cache(bt):
     assert torch.equal(out, out2)
 
 
-@pytest.mark.parametrize("L_B,P,hd,H", [(4, 1, 64, 8), (4, 2, 64, 8), (1, 1, 64, 3), (8, 2, 128, 4), (2, 4, 128, 16)])
+@pytest.mark.parametrize("L_B,P,hd,H", [
+    (4, 1, 64, 8), (4, 2, 64, 8), (1, 1, 64, 3), (8, 2, 128, 4), (2, 4, 128, 16),
+    # prefix length 8 (the longest of the prefix-length ablation): the block start is an 8-row causal step,
+    # the steps after it run over 8 .. 8 + L_B - 2 cached rows
+    (4, 8, 64, 4), (4, 8, 128, 3), (8, 8, 64, 2), (8, 8, 128, 2), (1, 8, 64, 5),
+    # local caches of 7, 8 and 9 rows at both head sizes (the deepest of the pipelined step kernels)
+    (8, 1, 128, 4), (6, 2, 128, 4), (6, 1, 128, 2), (8, 1, 64, 5), (6, 2, 64, 16)])
 def test_token_decoder_blocks(bt, L_B, P, hd, H):
     """Fused reset + append + local attention over several blocks; lengths, reset positions and
     cache rows bit-exact, outputs within tolerance."""
@@ -156,6 +162,54 @@ def test_token_masked_reset_attend_only_append_and_overflow(bt):
     st.zero_()
     bt.bt_token_decode_attn(cfg, lc, 0, to_dev(q), None, None, out, dev_status=st)
     assert not out.any() and st.item() == bt.BT_DEV_EMPTY
+
+
+@pytest.mark.parametrize("P,hd", [(2, 64), (4, 64), (2, 128), (4, 128), (8, 64)])
+def test_token_masked_reset_with_prefix_steps(bt, P, hd):
+    """Ragged batch (prompts whose partial last block was prefilled for some sequences while others
+    start a block): one call in which the sequences named by reset_mask drop their cache and take the P
+    prefix rows as a causal P-query step, while the others append the same number of rows to what
+    they hold - or are skipped, untouched and flagged, when those rows do not fit."""
+    B, H, L_B = 7, 4, 4
+    cap = P + L_B
+    cfg = bt.make_config(B, H, hd, L_B, P, 8, 2)
+    layer = 1
+    lc = bt.LocalCache(cfg)
+    lc.kv.copy_(to_dev(rnd(51, 1, tuple(lc.kv.shape))))
+    oc = oracle.Cache(B, H, cap, hd)
+    st = status_word()
+    # uneven starting lengths through single-row steps with a mask that keeps some sequences empty
+    lens0 = [0, 1, 2, 3, cap - P, cap - P + 1, cap]   # the last but one has no room for P more rows
+    for b, n in enumerate(lens0):
+        if n:
+            kb, vb = rnd(52, 10 + b, (1, H, n, hd)), rnd(52, 20 + b, (1, H, n, hd))
+            oc.k[b, :, :n], oc.v[b, :, :n] = kb[0], vb[0]
+            oc.len[b] = n
+    kv = np.zeros(tuple(lc.kv[layer].shape), np.uint16)
+    kv[:, :, :, 0], kv[:, :, :, 1] = oc.k, oc.v
+    lc.kv[layer].copy_(to_dev(kv))
+    lc.len[layer].copy_(torch.from_numpy(oc.len.copy()).cuda())
+    for step, mask in enumerate(([1, 0, 0, 1, 0, 0, 1], [0, 1, 0, 0, 1, 0, 0])):
+        mask = np.array(mask, np.uint8)
+        q, k, v = (rnd(53 + hd, 10 * step + i, (B, H, P, hd)) for i in range(3))
+        out = torch.full((B, H, P, hd), 3.0, dtype=torch.bfloat16, device="cuda")
+        before = gen.torch_to_bits(lc.kv[layer])
+        bt.bt_token_decode_attn(cfg, lc, layer, to_dev(q), to_dev(k), to_dev(v), out,
+                                reset_mask=torch.from_numpy(mask).cuda(), dev_status=st)
+        len_before = oc.len.copy()
+        ref = oracle.token_decode_attn(oc, q, k, v, reset_mask=mask)
+        assert_close(out, ref, f"masked reset, {P} rows, step {step}")
+        assert lc.len[layer].cpu().tolist() == oc.len.tolist()
+        gk, gv = local_kv_split(lc.kv[layer])
+        after = gen.torch_to_bits(lc.kv[layer])
+        for b in range(B):
+            n = oc.len[b]
+            assert np.array_equal(gk[b, :, :n], oc.k[b, :, :n]) and np.array_equal(gv[b, :, :n], oc.v[b, :, :n])
+            skipped = not mask[b] and len_before[b] + P > cap
+            if skipped:  # no room: nothing written, zeros out
+                assert np.array_equal(after[b], before[b]) and not out[b].any() and oc.len[b] == len_before[b]
+    assert st.item() == bt.BT_DEV_OVERFLOW == int(oc.status[0])
+    assert not lc.len[0].any()
 
 
 # ------------------------------------------------------------------ block decode: tiles, tails, splits
@@ -269,7 +323,7 @@ def test_l_b_one_block_decoder_is_vanilla_causal_attention(bt):
 
 @pytest.mark.parametrize("plain", [0, 1])
 @pytest.mark.parametrize("hd,T,B,H", [(128, 128, 2, 2), (128, 300, 1, 3), (64, 257, 2, 2), (128, 512, 1, 2), (64, 33, 3, 1),
-                                      (128, 1, 1, 1), (64, 640, 1, 2), (128, 1024, 1, 1)])
+                                      (128, 1, 1, 1), (64, 640, 1, 2), (128, 1024, 1, 1), (128, 2048, 1, 2), (64, 2048, 1, 1)])
 def test_block_prefill_shapes(bt, hd, T, B, H, plain):
     cfg = bt.make_config(B, H, hd, 4, 1, T, 1, prefill_plain=plain)
     q, k, v = (rnd(100 + T, i, (B, H, T, hd)) for i in range(3))
