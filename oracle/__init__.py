@@ -135,15 +135,14 @@ def local_kv_reset(c: Cache, mask=None):
 
 
 def token_decode_attn(c: Cache, q, k_new, v_new, reset_first=False, reset_mask=None, scale=None, f32=False):
-    """Fused token-decoder step: reset? -> append n_q rows -> causal attention inside the block."""
+    """Fused token-decoder step: reset? -> append n_q rows -> causal attention inside the block.
+    k_new = v_new = None: nothing is appended, the n_q queries belong to the last n_q cached rows."""
     q = _u16(q)
     n_q = q.shape[2]
     assert q.shape == (c.B, c.H, n_q, c.hd)
     if k_new is not None:
         k_new, v_new = _u16(k_new), _u16(v_new)
         assert k_new.shape == q.shape and v_new.shape == q.shape
-    else:
-        assert n_q == 1
     m = None if reset_mask is None else np.ascontiguousarray(reset_mask, np.uint8)
     dt, sfx = _real(f32)
     out = np.zeros((c.B, c.H, n_q, c.hd), dt)
@@ -189,3 +188,53 @@ def block_prefill_attn(q, k, v, scale=None, f32=False, kv_seq_stride=None):
         B, H, T, hd, _p(q), _p(k), _p(v), ctypes.c_longlong(stride),
         ctypes.c_double(scale if scale is not None else default_scale(hd)), _p(out))
     return out
+
+
+def linear(x, W, bias=None, f32=False):
+    """y = W x + b over rows: x [M,K], W [N,K] (row o = weights of output feature o), bias [N] -> [M,N]."""
+    x, W = _u16(x), _u16(W)
+    M, K = x.shape
+    N = W.shape[0]
+    assert W.shape == (N, K)
+    if bias is not None:
+        bias = _u16(bias)
+        assert bias.shape == (N,)
+    dt, sfx = _real(f32)
+    y = np.zeros((M, N), dt)
+    getattr(lib(), "bto_linear" + sfx)(M, K, N, _p(x), _p(W), _p(bias), _p(y))
+    return y
+
+
+def round_to_bf16(v):
+    """Nearest bf16 (ties to even) of float64 values, as uint16 bits."""
+    f = lib().bto_round_to_bf16
+    f.restype, f.argtypes = ctypes.c_uint16, [ctypes.c_double]
+    a = np.asarray(v, np.float64)
+    return np.array([f(float(t)) for t in a.ravel()], np.uint16).reshape(a.shape)
+
+
+def prefix_project(ctx, W, bias, P, f32=False):
+    """Context embedding -> P prefix token embeddings (section 2.4; appendix on token-decoder variants,
+    "Prefix"): ctx [B,D], W [P*D,D], bias [P*D] or None -> [B,P,D] (output feature p*D + d is
+    dimension d of prefix token p)."""
+    B, D = ctx.shape
+    assert W.shape == (P * D, D)
+    return linear(ctx, W, bias, f32=f32).reshape(B, P, D)
+
+
+def qkv_project_append(c: Cache, x, W, bias=None, reset_first=False, reset_mask=None, f32=False):
+    """y = W x + b for x [B,n,D]; returns q [B,H,n,hd] (not rounded) and appends the K and V parts,
+    rounded to bf16, to the cache (block or local) as kv_append would, after the optional reset."""
+    x, W = _u16(x), _u16(W)
+    B, n, D = x.shape
+    assert B == c.B and D == c.H * c.hd and W.shape == (3 * D, D)
+    if bias is not None:
+        bias = _u16(bias)
+        assert bias.shape == (3 * D,)
+    m = None if reset_mask is None else np.ascontiguousarray(reset_mask, np.uint8)
+    dt, sfx = _real(f32)
+    q = np.zeros((B, c.H, n, c.hd), dt)
+    getattr(lib(), "bto_qkv_project_append" + sfx)(
+        B, n, c.H, c.hd, c.cap, _p(x), _p(W), _p(bias), _p(c.k), _p(c.v), _p(c.len),
+        ctypes.c_int(1 if reset_first else 0), _p(m), _p(q), _p(c.status))
+    return q

@@ -16,7 +16,12 @@
  *     block decoded so far; its cache is dropped at each block boundary;
  *   - attention itself is softmax(scale * q.K^T) V, written here as the textbook
  *     two-pass formula: scores, max, exponentials, sums, divide.  No tiling, no
- *     running rescale, no splitting of the row range.
+ *     running rescale, no splitting of the row range;
+ *   - the linear maps either side of that path (section 2.4 and the appendix on
+ *     token-decoder variants: the context embedding is projected into P prefix token
+ *     embeddings; sections 2.1 and 2.3: each layer caches the K,V it computes from
+ *     its input) are y = W x + b as a triple loop, and "project, then cache" is that
+ *     product followed by the ordinary append.
  *
  * Precision: the file is compiled twice.  REAL=double gives the primary oracle
  * (symbols bto_*), REAL=float gives a single-precision twin (bto_*_f32) used to
@@ -31,7 +36,10 @@
  * pure Python on tiny inputs, the library routine for scaled-dot-product
  * attention in float64, L_B = 1 equals vanilla causal attention, cached decode
  * equals the matching row of the full recompute, no dependence on other blocks,
- * the integer schedule model, and planted-mistake tests.
+ * the integer schedule model, and planted-mistake tests.  The projections: identity
+ * and one-hot weights give back rows of the input bit for bit, numpy's float64
+ * matrix product, zero input gives the bias, and "project-then-append" equals
+ * kv_append of separately projected, separately rounded rows.
  */
 #include <math.h>
 #include <stdint.h>
@@ -174,8 +182,10 @@ void FN(bto_local_kv_reset)(int B, int32_t* len, const uint8_t* mask)
  * itself.  Nothing outside the block is visible.  n_q = 1 for a token step;
  * n_q = P at a block start appends the prefix rows with a causal mask among them
  * (the token decoder is an autoregressive transformer).
- * With k_new == NULL nothing is appended and the single query (n_q must be 1)
- * attends to rows 0..len-1.
+ * With k_new == NULL nothing is appended: the n_q queries are those of the last
+ * n_q rows already in the cache (written there by the projection that cached
+ * them), so query i attends to rows 0..len-n_q+i - the same causal rule, counted
+ * from the end; n_q = 1 attends to rows 0..len-1.
  * q, k_new, v_new: [B][H][n_q][hd]; out: [B][H][n_q][hd]; cache [B][H][cap][hd].
  * Overflow: sequence skipped (no write, zeros out, ST_OVERFLOW).  Attend-only on
  * an empty cache: zeros and ST_EMPTY.
@@ -208,7 +218,7 @@ void FN(bto_token_decode_attn)(int B, int H, int hd, int cap, uint16_t* kc, uint
                         memcpy(Vb + (size_t)(len_old + i) * hd, v_new + (bh * n_q + i) * hd, sizeof(uint16_t) * (size_t)hd);
                     }
                 for (int i = 0; i < n_q; ++i) {
-                    int n = appended ? len_old + i + 1 : len_old;
+                    int n = appended ? len_old + i + 1 : len_old - n_q + i + 1;
                     if (n <= 0) st |= ST_EMPTY;
                     attend_rows(q + (bh * n_q + i) * hd, Kb, Vb, n, hd, (REAL)scale, out + (bh * n_q + i) * hd, NULL);
                 }
@@ -239,4 +249,74 @@ void FN(bto_block_prefill_attn)(int B, int H, int T, int hd, const uint16_t* q, 
             attend_rows(q + ((size_t)bh * T + t) * hd, Kb, Vb, t + 1, hd, (REAL)scale,
                         out + ((size_t)bh * T + t) * hd, NULL);
         }
+}
+
+/*
+ * Linear map y = W x + b over M rows (the appendix on token-decoder variants, "Prefix": the
+ * context embedding is projected into prefix token embeddings; any nn.Linear-shaped layer).
+ * x: [M][K] bf16 bits; W: [N][K] bf16 bits (row o holds the weights of output feature o);
+ * bias: [N] bf16 bits or NULL; y: [M][N] REAL, not rounded.
+ */
+void FN(bto_linear)(int M, int K, int N, const uint16_t* x, const uint16_t* W, const uint16_t* bias, REAL* y)
+{
+#pragma omp parallel for schedule(static)
+    for (int m = 0; m < M; ++m)
+        for (int o = 0; o < N; ++o) {
+            REAL acc = bias ? widen(bias[o]) : (REAL)0;
+            for (int k = 0; k < K; ++k) acc += widen(x[(size_t)m * K + k]) * widen(W[(size_t)o * K + k]);
+            y[(size_t)m * N + o] = acc;
+        }
+}
+
+/* Nearest bf16 (ties to even) of a finite REAL, as bits; bf16 keeps 8 significant bits. */
+static uint16_t round_to_bf16(REAL v)
+{
+    double a = fabs((double)v);
+    if (a == 0) return signbit((double)v) ? 0x8000u : 0;
+    int e = ilogb(a);                     /* 2^e <= a < 2^(e+1) */
+    if (e < -126) e = -126;               /* subnormal range: fixed spacing */
+    double q = nearbyint(ldexp(a, 7 - e)); /* default rounding mode: ties to even */
+    float f = (float)ldexp(q, e - 7);     /* exactly representable */
+    uint32_t u;
+    memcpy(&u, &f, sizeof u);
+    return (uint16_t)((u >> 16) | (signbit((double)v) ? 0x8000u : 0));
+}
+uint16_t FN(bto_round_to_bf16)(double v) { return round_to_bf16((REAL)v); }
+
+/*
+ * QKV projection whose K,V go straight into a cache (sections 2.1 and 2.3: the K,V of every
+ * processed block are cached; section 2.4: likewise for the rows of the current block in the
+ * local cache).  x: [B][n][D] bf16 bits, D = H*hd; W: [3D][D] with output features ordered
+ * Q (h*hd+d), then K, then V; bias [3D] or NULL.
+ *   y = W x + b  per row;  q_out[b][h][i][d] = y_Q (REAL, not rounded);
+ *   the K and V parts, rounded to bf16 (the cache's storage type), are appended to sequence b's
+ *   cache at rows len[b]..len[b]+n-1 exactly as bto_kv_append does, after the optional reset
+ *   (reset_mask ? reset_mask[b] : reset_first) that bto_token_decode_attn also knows.
+ * A sequence without room keeps its cache and length (ST_OVERFLOW); its q is still produced.
+ */
+void FN(bto_qkv_project_append)(int B, int n, int H, int hd, int cap, const uint16_t* x, const uint16_t* W,
+                                const uint16_t* bias, uint16_t* kc, uint16_t* vc, int32_t* len, int reset_first,
+                                const uint8_t* reset_mask, REAL* q_out, uint32_t* status)
+{
+    const int D = H * hd;
+    REAL* y = (REAL*)malloc(sizeof(REAL) * (size_t)B * n * 3 * D);
+    FN(bto_linear)(B * n, D, 3 * D, x, W, bias, y);
+    uint16_t* k_new = (uint16_t*)malloc(sizeof(uint16_t) * (size_t)B * n * D);
+    uint16_t* v_new = (uint16_t*)malloc(sizeof(uint16_t) * (size_t)B * n * D);
+    for (int b = 0; b < B; ++b)
+        for (int i = 0; i < n; ++i)
+            for (int h = 0; h < H; ++h)
+                for (int d = 0; d < hd; ++d) {
+                    const REAL* row = y + ((size_t)b * n + i) * 3 * D;
+                    size_t o = ((((size_t)b * H + h) * n) + i) * hd + d;   /* [B][H][n][hd] */
+                    q_out[o] = row[h * hd + d];
+                    k_new[o] = round_to_bf16(row[D + h * hd + d]);
+                    v_new[o] = round_to_bf16(row[2 * D + h * hd + d]);
+                }
+    for (int b = 0; b < B; ++b)
+        if (reset_mask ? (reset_mask[b] != 0) : (reset_first != 0)) len[b] = 0;
+    FN(bto_kv_append)(B, H, hd, cap, kc, vc, len, k_new, v_new, n, status);
+    free(y);
+    free(k_new);
+    free(v_new);
 }

@@ -22,8 +22,24 @@ MUTANTS = {
     "causal_sees_one_ahead": ("Kb, Vb, t + 1, hd", "Kb, Vb, (t + 2 > T ? T : t + 2), hd"),
     "decode_drops_last_row": ("int n = len[b];", "int n = len[b] - 1;"),
     "decode_reads_one_past": ("int n = len[b];", "int n = len[b] + 1;"),
-    "token_excludes_itself": ("int n = appended ? len_old + i + 1 : len_old;",
-                              "int n = appended ? len_old + i : len_old;"),
+    "token_excludes_itself": ("int n = appended ? len_old + i + 1 : len_old - n_q + i + 1;",
+                              "int n = appended ? len_old + i : len_old - n_q + i + 1;"),
+    "attend_only_not_causal": ("int n = appended ? len_old + i + 1 : len_old - n_q + i + 1;",
+                               "int n = appended ? len_old + i + 1 : len_old;"),
+    "attend_only_counts_from_the_start": ("int n = appended ? len_old + i + 1 : len_old - n_q + i + 1;",
+                                          "int n = appended ? len_old + i + 1 : i + 1;"),
+    "linear_weight_transposed": ("widen(W[(size_t)o * K + k])", "widen(W[((size_t)k * N + o) % ((size_t)N * K)])"),
+    "linear_bias_dropped": ("REAL acc = bias ? widen(bias[o]) : (REAL)0;", "REAL acc = 0;"),
+    "linear_bias_of_wrong_feature": ("REAL acc = bias ? widen(bias[o]) : (REAL)0;", "REAL acc = bias ? widen(bias[(o + 1) % N]) : (REAL)0;"),
+    "rounding_truncates": ("double q = nearbyint(ldexp(a, 7 - e));", "double q = floor(ldexp(a, 7 - e));"),
+    "rounding_ties_away": ("double q = nearbyint(ldexp(a, 7 - e));", "double q = floor(ldexp(a, 7 - e) + 0.5);"),
+    "projection_k_and_v_swapped": ("k_new[o] = round_to_bf16(row[D + h * hd + d]);\n                    v_new[o] = round_to_bf16(row[2 * D + h * hd + d]);",
+                                   "k_new[o] = round_to_bf16(row[2 * D + h * hd + d]);\n                    v_new[o] = round_to_bf16(row[D + h * hd + d]);"),
+    "projection_q_not_grouped_by_head": ("size_t o = ((((size_t)b * H + h) * n) + i) * hd + d;   /* [B][H][n][hd] */",
+                                         "size_t o = ((((size_t)b * n + i) * H) + h) * hd + d;"),
+    "projection_takes_k_for_q": ("q_out[o] = row[h * hd + d];", "q_out[o] = row[D + h * hd + d];"),
+    "projection_reset_ignored": ("if (reset_mask ? (reset_mask[b] != 0) : (reset_first != 0)) len[b] = 0;\n    FN(bto_kv_append)", ";\n    FN(bto_kv_append)"),
+    "projection_rows_of_wrong_token": ("const REAL* row = y + ((size_t)b * n + i) * 3 * D;", "const REAL* row = y + ((size_t)b * n + (n - 1 - i)) * 3 * D;"),
     "token_reset_ignored": ("if (do_reset) len[b] = 0;", ";"),
     "append_ignores_length": ("* cap + (size_t)(len[b] + i)) * hd;", "* cap + (size_t)(i)) * hd;"),
     "append_no_length_update": ("        len[b] += n_new;", "        ;"),
@@ -50,6 +66,14 @@ PIN_FUNCS = [
     lambda: pins.test_token_decoder_never_crosses_a_block_boundary(4, 2),
     pins.test_token_step_equals_attention_over_prefix_plus_same_block_tokens,
     pins.test_token_attend_only_and_masked_reset,
+    pins.test_attend_only_over_the_last_rows_equals_the_appending_step,
+    pins.test_round_to_bf16_is_nearest_even,
+    pins.test_linear_identity_one_hot_zero_input_and_library_product,
+    pins.test_prefix_projection_layout,
+    pins.test_qkv_projection_with_identity_blocks_caches_the_input_rows,
+    pins.test_project_then_append_equals_append_of_projected_rows,
+    pins.test_qkv_projection_reset_is_the_block_boundary_reset,
+    pins.test_projected_step_equals_appending_step_on_projected_rows,
 ]
 
 

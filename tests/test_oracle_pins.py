@@ -381,6 +381,169 @@ def test_token_overflow_is_skipped_and_flagged():
     assert not out[1].any() and not c.k[1].any()
 
 
+def test_attend_only_over_the_last_rows_equals_the_appending_step():
+    """k_new = None with n_q queries: they belong to the last n_q cached rows, query i sees rows
+    0 .. len - n_q + i.  Pinned to the appending form of the same step, which the pins above fix."""
+    B, H, hd, cap = 3, 2, 8, 9
+    for n_q, start in ((1, 3), (2, 0), (4, 2), (4, 5)):
+        a = oracle.Cache(B, H, cap, hd)
+        a.k[...], a.v[...] = rnd(24, 1, a.k.shape), rnd(24, 2, a.v.shape)
+        a.len[...] = start
+        b = a.copy()
+        q, k, v = (rnd(24, 10 * n_q + i, (B, H, n_q, hd)) for i in range(3))
+        want = oracle.token_decode_attn(a, q, k, v)
+        oracle.kv_append(b, k, v)
+        got = oracle.token_decode_attn(b, q, None, None)
+        assert np.array_equal(got, want) and b.len.tolist() == a.len.tolist() == [start + n_q] * B
+        # and to the library routine: query i over the first start + i + 1 rows
+        for i in range(n_q):
+            m = start + i + 1
+            np.testing.assert_allclose(got[:, :, i:i + 1], sdpa64(q[:, :, i:i + 1], b.k[:, :, :m], b.v[:, :, :m], False),
+                                       rtol=0, atol=1e-12)
+    # fewer rows than queries: the leading queries have nothing to see
+    e = oracle.Cache(1, 1, 4, hd)
+    e.k[...], e.v[...] = rnd(24, 5, e.k.shape), rnd(24, 6, e.v.shape)
+    e.len[...] = 1
+    out = oracle.token_decode_attn(e, rnd(24, 7, (1, 1, 2, hd)), None, None)
+    assert not out[0, 0, 0].any() and np.array_equal(out[0, 0, 1], widen(e.v[0, 0, 0])) and e.status[0] & oracle.ST_EMPTY
+
+
+# ---------------------------------------------------------------- projections either side of the path
+
+def test_round_to_bf16_is_nearest_even():
+    # ties: 1 + 2^-8 lies midway between 1 (even mantissa) and 1 + 2^-7; 1 + 3*2^-8 between 1 + 2^-7 (odd) and 1 + 2^-6
+    cases = {1.0: 0x3F80, 1.0 + 2.0 ** -8: 0x3F80, 1.0 + 3 * 2.0 ** -8: 0x3F82, 1.0 + 2.0 ** -8 + 2.0 ** -30: 0x3F81,
+             -2.5: 0xC020, 0.0: 0x0000, 255.5: 0x4380, 3.0e-5: int(bits([3.0e-5])[0])}
+    for v, want in cases.items():
+        assert int(oracle.round_to_bf16([v])[0]) == want, v
+    # every float32 input: the independent float32 -> bf16 rounding of the input generators agrees
+    x = np.concatenate([widen(rnd(30, 0, (4096,))) * s for s in (1.0, 37.0, 1e-3)]).astype(np.float32)
+    x = (x.astype(np.float64) * (1.0 + 2.0 ** -10)).astype(np.float32)  # off the bf16 grid
+    assert np.array_equal(oracle.round_to_bf16(x.astype(np.float64)), bits(x))
+
+
+def test_linear_identity_one_hot_zero_input_and_library_product():
+    M, K = 5, 12
+    x = rnd(31, 0, (M, K))
+    eye = bits(np.eye(K))
+    assert np.array_equal(oracle.linear(x, eye), widen(x))                      # identity: rows come back exactly
+    perm = np.random.default_rng(31).permutation(K)
+    onehot = bits(2.0 * np.eye(K)[perm])                                        # output o = 2 * x[perm[o]]
+    assert np.array_equal(oracle.linear(x, onehot), 2.0 * widen(x)[:, perm])
+    W, b = rnd(31, 1, (7, K)), rnd(31, 2, (7,))
+    assert np.array_equal(oracle.linear(bits(np.zeros((M, K))), W, b), np.tile(widen(b), (M, 1)))   # zero input: the bias
+    ref = widen(x) @ widen(W).T + widen(b)                                      # numpy's float64 product
+    np.testing.assert_allclose(oracle.linear(x, W, b), ref, rtol=0, atol=1e-12)
+    np.testing.assert_allclose(oracle.linear(x, W), ref - widen(b), rtol=0, atol=1e-12)
+    np.testing.assert_allclose(oracle.linear(x, W, b, f32=True), ref, rtol=0, atol=2e-5)
+    # a non-square, non-symmetric case told apart from its transpose: W[o][k] = 1 only at (0, 1)
+    W2 = np.zeros((3, 2)); W2[0, 1] = 1.0
+    y = oracle.linear(bits([[5.0, 7.0]]), bits(W2))
+    assert y.tolist() == [[7.0, 0.0, 0.0]]
+
+
+def test_prefix_projection_layout():
+    """Output feature p*D + d is dimension d of prefix token p (section 2.4: the context embedding is
+    projected into P prefix token embeddings)."""
+    B, D, P = 3, 8, 2
+    ctx = rnd(32, 0, (B, D))
+    W = np.zeros((P * D, D))
+    W[:D] = np.eye(D)                 # prefix token 0 = the context embedding
+    W[D:] = -np.eye(D)[::-1]          # prefix token 1 = its negated mirror image
+    out = oracle.prefix_project(ctx, bits(W), None, P)
+    assert out.shape == (B, P, D)
+    assert np.array_equal(out[:, 0], widen(ctx)) and np.array_equal(out[:, 1], -widen(ctx)[:, ::-1])
+    b = rnd(32, 1, (P * D,))
+    np.testing.assert_allclose(oracle.prefix_project(ctx, bits(W), b, P), out + widen(b).reshape(1, P, D), rtol=0, atol=1e-12)
+
+
+def _qkv_case(seed, B, n, H, hd, cap, lens):
+    D = H * hd
+    c = oracle.Cache(B, H, cap, hd)
+    c.k[...], c.v[...] = rnd(seed, 1, c.k.shape), rnd(seed, 2, c.v.shape)
+    c.len[...] = lens
+    return c, rnd(seed, 3, (B, n, D)), D
+
+
+def test_qkv_projection_with_identity_blocks_caches_the_input_rows():
+    """W = [I; 2I; -I]: q is x regrouped by head, the K rows are 2x and the V rows -x, bit for bit, at
+    rows len .. len+n-1 of each head's slab; a sequence without room keeps everything."""
+    B, n, H, hd, cap = 4, 3, 2, 4, 6
+    lens = [0, 2, 3, 4]                      # the last one has no room for 3 more rows
+    c, x, D = _qkv_case(33, B, n, H, hd, cap, lens)
+    before = c.copy()
+    W = bits(np.concatenate([np.eye(D), 2 * np.eye(D), -np.eye(D)]))
+    q = oracle.qkv_project_append(c, x, W)
+    xr = x.reshape(B, n, H, hd).transpose(0, 2, 1, 3)          # [B,H,n,hd]
+    assert np.array_equal(q, widen(xr))
+    assert c.len.tolist() == [3, 5, 6, 4] and c.status[0] == oracle.ST_OVERFLOW
+    for b in range(3):
+        l = lens[b]
+        assert np.array_equal(c.k[b, :, l:l + n], bits(2.0 * widen(xr[b]))) and np.array_equal(c.v[b, :, l:l + n], bits(-widen(xr[b])))
+        assert np.array_equal(c.k[b, :, :l], before.k[b, :, :l]) and np.array_equal(c.k[b, :, l + n:], before.k[b, :, l + n:])
+    assert np.array_equal(c.k[3], before.k[3]) and np.array_equal(c.v[3], before.v[3])
+
+
+def test_project_then_append_equals_append_of_projected_rows():
+    B, n, H, hd, cap = 3, 2, 3, 8, 7
+    c, x, D = _qkv_case(34, B, n, H, hd, cap, [0, 5, 1])
+    W, bias = rnd(34, 4, (3 * D, D)), rnd(34, 5, (3 * D,))
+    ref = c.copy()
+    q = oracle.qkv_project_append(c, x, W, bias)
+    y = (widen(x).reshape(B * n, D) @ widen(W).T + widen(bias)).reshape(B, n, 3, H, hd)   # numpy's float64 product
+    np.testing.assert_allclose(q, y[:, :, 0].transpose(0, 2, 1, 3), rtol=0, atol=1e-12)
+    kn, vn = (np.ascontiguousarray(y[:, :, j].transpose(0, 2, 1, 3)) for j in (1, 2))
+    oracle.kv_append(ref, oracle.round_to_bf16(kn), oracle.round_to_bf16(vn))
+    # (the two float64 sums may differ in the last place, which can move a value across a rounding boundary)
+    for got, want in ((c.k, ref.k), (c.v, ref.v)):
+        d = np.abs(got.astype(np.int32) - want.astype(np.int32))
+        assert d.max() <= 1 and (d > 0).mean() < 1e-3
+    assert np.array_equal(c.len, ref.len) and c.len.tolist() == [2, 7, 3]
+    # exact arithmetic (small integers): no rounding anywhere, so the rows are fixed bit for bit
+    rng = np.random.default_rng(34)
+    xi, Wi = bits(rng.integers(-1, 2, (B, n, D))), bits(rng.integers(-1, 3, (3 * D, D)))
+    c2, r2 = oracle.Cache(B, H, cap, hd), oracle.Cache(B, H, cap, hd)
+    oracle.qkv_project_append(c2, xi, Wi)
+    yi = (widen(xi).reshape(B * n, D) @ widen(Wi).T).reshape(B, n, 3, H, hd)
+    oracle.kv_append(r2, *(bits(np.ascontiguousarray(yi[:, :, j].transpose(0, 2, 1, 3))) for j in (1, 2)))
+    assert np.array_equal(c2.k, r2.k) and np.array_equal(c2.v, r2.v) and c2.len.tolist() == [n] * B
+
+
+def test_qkv_projection_reset_is_the_block_boundary_reset():
+    B, n, H, hd, cap = 4, 2, 2, 4, 5
+    c, x, D = _qkv_case(35, B, n, H, hd, cap, [3, 4, 0, 5])
+    W = rnd(35, 4, (3 * D, D))
+    a, b = c.copy(), c.copy()
+    mask = [1, 0, 0, 1]
+    qa = oracle.qkv_project_append(a, x, W, reset_mask=mask)
+    oracle.local_kv_reset(b, mask)
+    qb = oracle.qkv_project_append(b, x, W)
+    assert np.array_equal(qa, qb) and np.array_equal(a.k, b.k) and np.array_equal(a.v, b.v)
+    assert a.len.tolist() == b.len.tolist() == [2, 4, 2, 2] and a.status[0] == oracle.ST_OVERFLOW  # sequence 1: 4 + 2 > 5
+    e = c.copy()
+    oracle.qkv_project_append(e, x, W, reset_first=True)
+    assert e.len.tolist() == [2, 2, 2, 2] and e.status[0] == 0
+    # after a reset the rows land at index 0 .. n-1, as for the masked sequences above
+    assert np.array_equal(e.k[0, :, :n], a.k[0, :, :n]) and np.array_equal(e.v[3, :, :n], a.v[3, :, :n])
+
+
+def test_projected_step_equals_appending_step_on_projected_rows():
+    """The path with the projections in: project + cache, then attend-only over the cache, gives what the
+    fused append-and-attend step gives when handed the projected (rounded) rows."""
+    B, n, H, hd, cap = 2, 2, 2, 8, 6
+    c, x, D = _qkv_case(36, B, n, H, hd, cap, [1, 3])
+    W = rnd(36, 4, (3 * D, D))
+    a = c.copy()
+    q = oracle.qkv_project_append(c, x, W)
+    qb = oracle.round_to_bf16(q)
+    got = oracle.token_decode_attn(c, qb, None, None)
+    l0 = a.len.copy()
+    kn = np.stack([c.k[b, :, l0[b]:l0[b] + n] for b in range(B)])
+    vn = np.stack([c.v[b, :, l0[b]:l0[b] + n] for b in range(B)])
+    want = oracle.token_decode_attn(a, qb, kn, vn)
+    assert np.array_equal(got, want)
+
+
 # ---------------------------------------------------------------- schedule model + byte model
 
 def golden():
