@@ -223,8 +223,10 @@ bt_status bt_local_kv_append(const bt_config* cfg, bt_local_cache* cache, int la
  *      the earlier tokens of the same block and itself - never anything outside the block;
  *   4. len[b] += n_q.
  * n_q = 1 for a token step; n_q = P at a block start appends the P prefix rows, causally
- * masked among themselves.  k_new == v_new == NULL: nothing is appended, n_q must be 1 and
- * the query attends to rows 0 .. len[b]-1 (zeros and BT_DEV_EMPTY if there are none).
+ * masked among themselves.  k_new == v_new == NULL: nothing is appended (the rows were cached
+ * by bt_local_qkv_project_append); the n_q queries are those of the last n_q cached rows, so
+ * query i attends to rows 0 .. len[b]-n_q+i - with n_q = 1, rows 0 .. len[b]-1 (zeros and
+ * BT_DEV_EMPTY for a query with no row to see).
  * A sequence without room for n_q rows is skipped: nothing written, zeros out,
  * BT_DEV_OVERFLOW.  q, out: [B][H][n_q][hd].
  */
@@ -262,6 +264,48 @@ bt_status bt_block_decode_step_host(const bt_config* cfg, bt_block_cache* cache,
                                     void* out_host, void* q_dev, void* k_dev, void* v_dev, void* out_dev,
                                     void* workspace, size_t workspace_bytes, uint32_t* dev_status,
                                     void* stream);
+
+/*
+ * Prefix projection (section 2.4; appendix on token-decoder variants, "Prefix"): the context embedding
+ * the block decoder produced for a block is projected into the P = cfg->prefix_len prefix token
+ * embeddings that seed the token decoder:
+ *   prefix_out[b][p][:] = W_p ctx[b][:] + bias_p,   p < P.
+ * ctx: bf16 [B][D], D = H * hd.  w_prefix: bf16 [P*D][D], row p*D + d holds the weights of dimension d
+ * of prefix token p.  bias: bf16 [P*D] or NULL.  prefix_out: bf16 [B][P][D].  A dense product on the
+ * tensor cores (TMA-fed tcgen05 MMA, fp32 accumulation in tensor memory), results rounded to bf16.
+ * dev_status: BT_DEV_TIMEOUT if a (bounded) wait inside the kernel ran out.
+ */
+bt_status bt_prefix_project(const bt_config* cfg, const void* ctx, const void* w_prefix, const void* bias,
+                            void* prefix_out, uint32_t* dev_status, void* stream);
+
+/*
+ * QKV projection whose K and V go straight into the cache (sections 2.1 and 2.3: the K,V of every
+ * processed block are cached; section 2.4: likewise the rows of the current block, locally), so that
+ * no separate append pass reads and writes them again.  x: bf16 [B][n_rows][D], the layer's input for
+ * the n_rows new positions of every sequence (one block embedding; P prefix embeddings; one token).
+ * w_qkv: bf16 [3*D][D], output features ordered Q, K, V and (head, dim) inside each; bias: bf16 [3*D]
+ * or NULL.  With y = w_qkv x + bias per row (fp32 accumulation, rounded to bf16):
+ *   q_out[b][h][i][:] = the Q part of row i              (bf16 [B][H][n_rows][hd], the layout the
+ *                                                         attention calls take)
+ *   cache rows len[b]+i of head h = the K and V parts,   i < n_rows
+ *   len[b] += n_rows.
+ * A sequence without room for n_rows more rows keeps its cache and length, BT_DEV_OVERFLOW is raised
+ * (its q_out rows are still written).  Two launches: the product with the cache-writing epilogue, then
+ * a small one that advances the lengths once every tile has read the old ones.
+ * Attention then runs over the cache as it stands: bt_block_decode_attn for the block decoder,
+ * bt_token_decode_attn with k_new = v_new = NULL (n_q = n_rows) for the token decoder.
+ * Returns BT_ERR_CAPACITY if n_rows exceeds the cache capacity.
+ *
+ * The local form adds the block-boundary reset of bt_token_decode_attn: where
+ * (reset_mask ? reset_mask[b] : reset_first) holds, sequence b's rows land at index 0 .. n_rows-1
+ * and its length becomes n_rows.
+ */
+bt_status bt_block_qkv_project_append(const bt_config* cfg, bt_block_cache* cache, int layer, const void* x,
+                                      int n_rows, const void* w_qkv, const void* bias, void* q_out,
+                                      uint32_t* dev_status, void* stream);
+bt_status bt_local_qkv_project_append(const bt_config* cfg, bt_local_cache* cache, int layer, const void* x,
+                                      int n_rows, const void* w_qkv, const void* bias, int reset_first,
+                                      const uint8_t* reset_mask, void* q_out, uint32_t* dev_status, void* stream);
 
 /*
  * Self-test of the bounded waits (test support; the paper has no counterpart).  Every wait inside the

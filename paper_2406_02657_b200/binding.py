@@ -22,6 +22,7 @@ EXPORTS = [
     "bt_block_decode_attn", "bt_local_kv_reset", "bt_local_kv_append", "bt_token_decode_attn",
     "bt_block_prefill_attn", "bt_block_decode_step_host", "bt_block_decode_attn_noalloc",
     "bt_workspace_init", "bt_block_decode_step", "bt_block_decode_step_multi", "bt_selftest_bounded_wait",
+    "bt_prefix_project", "bt_block_qkv_project_append", "bt_local_qkv_project_append",
 ]
 
 
@@ -73,6 +74,9 @@ def _load() -> ctypes.CDLL:
                                               vp, vp, vp, vp, vp, u64, vp, vp]
     lib.bt_block_decode_attn_noalloc.argtypes = [cfgp, ctypes.POINTER(bt_block_cache), i32, vp, vp, vp, vp]
     lib.bt_selftest_bounded_wait.argtypes = [vp, vp, vp]
+    lib.bt_prefix_project.argtypes = [cfgp, vp, vp, vp, vp, vp, vp]
+    lib.bt_block_qkv_project_append.argtypes = [cfgp, ctypes.POINTER(bt_block_cache), i32, vp, i32, vp, vp, vp, vp, vp]
+    lib.bt_local_qkv_project_append.argtypes = [cfgp, ctypes.POINTER(bt_local_cache), i32, vp, i32, vp, vp, i32, vp, vp, vp, vp]
     for name in EXPORTS[4:]:
         getattr(lib, name).restype = ctypes.c_int
     return lib
@@ -200,6 +204,30 @@ def bt_block_decode_attn_noalloc(cfg, cache: BlockCache, layer, q, out, dev_stat
     BT_STATIC_WORKSPACE_BYTES; calls on one device share the scratch, so do not overlap them."""
     _check(_lib.bt_block_decode_attn_noalloc(ctypes.byref(cfg), ctypes.byref(cache.c), layer, _ptr(q), _ptr(out),
                                              _ptr(dev_status), _stream(stream)), "bt_block_decode_attn_noalloc")
+
+
+def bt_prefix_project(cfg, ctx, w_prefix, bias, prefix_out, dev_status=None, stream=None):
+    """Context embedding [B,D] -> P prefix token embeddings [B,P,D]."""
+    _check(_lib.bt_prefix_project(ctypes.byref(cfg), _ptr(ctx), _ptr(w_prefix), _ptr(bias), _ptr(prefix_out),
+                                  _ptr(dev_status), _stream(stream)), "bt_prefix_project")
+
+
+def bt_block_qkv_project_append(cfg, cache: BlockCache, layer, x, w_qkv, bias, q_out, n_rows=None, dev_status=None, stream=None):
+    """QKV projection of x [B,n,D]; Q -> q_out [B,H,n,hd], K and V rows appended to the block cache."""
+    n_rows = x.shape[1] if n_rows is None else n_rows
+    _check(_lib.bt_block_qkv_project_append(ctypes.byref(cfg), ctypes.byref(cache.c), layer, _ptr(x), n_rows, _ptr(w_qkv),
+                                            _ptr(bias), _ptr(q_out), _ptr(dev_status), _stream(stream)),
+           "bt_block_qkv_project_append")
+
+
+def bt_local_qkv_project_append(cfg, cache: LocalCache, layer, x, w_qkv, bias, q_out, n_rows=None, reset_first=False,
+                                reset_mask=None, dev_status=None, stream=None):
+    """QKV projection of x [B,n,D]; Q -> q_out [B,H,n,hd], K and V rows appended to the local cache
+    (after the optional block-boundary reset)."""
+    n_rows = x.shape[1] if n_rows is None else n_rows
+    _check(_lib.bt_local_qkv_project_append(ctypes.byref(cfg), ctypes.byref(cache.c), layer, _ptr(x), n_rows, _ptr(w_qkv),
+                                            _ptr(bias), 1 if reset_first else 0, _ptr(reset_mask), _ptr(q_out),
+                                            _ptr(dev_status), _stream(stream)), "bt_local_qkv_project_append")
 
 
 def bt_selftest_bounded_wait(report, dev_status, stream=None):

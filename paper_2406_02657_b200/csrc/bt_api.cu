@@ -296,7 +296,6 @@ bt_status bt_token_decode_attn(const bt_config* cfg, bt_local_cache* cache, int 
     if (!cache || !cache->kv || !cache->len || !q || !out) return BT_ERR_NULL;
     if ((k_new == nullptr) != (v_new == nullptr)) return BT_ERR_NULL;
     if (n_q <= 0) return BT_ERR_SHAPE;
-    if (!k_new && n_q != 1) return BT_ERR_SHAPE;
     if (n_q > local_cap(cfg)) return BT_ERR_CAPACITY;
     if (!local_cache_aligned(cache) || !al16(q) || !al16(k_new) || !al16(v_new) || !al16(out) || !al4(dev_status))
         return BT_ERR_UNSUPPORTED;
@@ -365,6 +364,95 @@ bt_status bt_block_decode_step_host(const bt_config* cfg, bt_block_cache* cache,
     if (st != BT_OK) return st;
     if (cudaMemcpyAsync(out_host, out_dev, bytes, cudaMemcpyDeviceToHost, s) != cudaSuccess) return BT_ERR_CUDA;
     return BT_OK;
+}
+
+// ---- the linear maps either side of the attention path
+
+static bt_status project_common(const bt_config* cfg, const void* x, const void* w, const void* bias, const void* out,
+                                const uint32_t* dev_status)
+{
+    if (!x || !w || !out) return BT_ERR_NULL;
+    if (!al16(x) || !al16(w) || !al16(bias) || !al16(out) || !al4(dev_status)) return BT_ERR_UNSUPPORTED;
+    if ((long long)cfg->heads * cfg->head_dim > (1 << 20)) return BT_ERR_UNSUPPORTED;
+    return BT_OK;
+}
+
+bt_status bt_prefix_project(const bt_config* cfg, const void* ctx, const void* w_prefix, const void* bias, void* prefix_out,
+                            uint32_t* dev_status, void* stream)
+{
+    bt_status st = check_config(cfg, 0);
+    if (st != BT_OK) return st;
+    st = project_common(cfg, ctx, w_prefix, bias, prefix_out, dev_status);
+    if (st != BT_OK) return st;
+    const long long D = (long long)cfg->heads * cfg->head_dim;
+    if (D * cfg->prefix_len > 0x7fffffffLL) return BT_ERR_UNSUPPORTED;
+    bt::ProjectArgs a = {};
+    a.x = ctx;
+    a.w = w_prefix;
+    a.bias = bias;
+    a.out = prefix_out;
+    a.M = cfg->batch;
+    a.K = (int)D;
+    a.N = (int)(D * cfg->prefix_len);
+    a.mode = bt::kProjectPlain;
+    a.dev_status = dev_status;
+    if (!bt::project_supported(a)) return BT_ERR_UNSUPPORTED;
+    return cuda_status(bt::launch_project(a, (cudaStream_t)stream));
+}
+
+static bt_status qkv_project(const bt_config* cfg, const bt::CacheView& view, const void* x, int n_rows, const void* w_qkv,
+                             const void* bias, int reset_first, const uint8_t* reset_mask, void* q_out, uint32_t* dev_status,
+                             void* stream)
+{
+    const long long D = (long long)cfg->heads * cfg->head_dim;
+    if ((long long)cfg->batch * n_rows > 0x7fffffffLL / 2 || 3 * D > 0x7fffffffLL) return BT_ERR_UNSUPPORTED;
+    bt::ProjectArgs a = {};
+    a.x = x;
+    a.w = w_qkv;
+    a.bias = bias;
+    a.out = q_out;
+    a.M = cfg->batch * n_rows;
+    a.K = (int)D;
+    a.N = (int)(3 * D);
+    a.mode = bt::kProjectQkv;
+    a.cache = view;
+    a.n_rows = n_rows;
+    a.H = cfg->heads;
+    a.hd = cfg->head_dim;
+    a.reset_first = reset_first ? 1 : 0;
+    a.reset_mask = reset_mask;
+    a.dev_status = dev_status;
+    if (!bt::project_supported(a)) return BT_ERR_UNSUPPORTED;
+    return cuda_status(bt::launch_project(a, (cudaStream_t)stream));
+}
+
+bt_status bt_block_qkv_project_append(const bt_config* cfg, bt_block_cache* cache, int layer, const void* x, int n_rows,
+                                      const void* w_qkv, const void* bias, void* q_out, uint32_t* dev_status, void* stream)
+{
+    bt_status st = check_config(cfg, layer);
+    if (st != BT_OK) return st;
+    if (!cache || !cache->k || !cache->v || !cache->len) return BT_ERR_NULL;
+    st = project_common(cfg, x, w_qkv, bias, q_out, dev_status);
+    if (st != BT_OK) return st;
+    if (n_rows <= 0) return BT_ERR_SHAPE;
+    if (n_rows > cfg->max_blocks) return BT_ERR_CAPACITY;
+    if (!block_cache_aligned(cache)) return BT_ERR_UNSUPPORTED;
+    return qkv_project(cfg, block_view(cfg, cache, layer), x, n_rows, w_qkv, bias, 0, nullptr, q_out, dev_status, stream);
+}
+
+bt_status bt_local_qkv_project_append(const bt_config* cfg, bt_local_cache* cache, int layer, const void* x, int n_rows,
+                                      const void* w_qkv, const void* bias, int reset_first, const uint8_t* reset_mask,
+                                      void* q_out, uint32_t* dev_status, void* stream)
+{
+    bt_status st = check_config(cfg, layer);
+    if (st != BT_OK) return st;
+    if (!cache || !cache->kv || !cache->len) return BT_ERR_NULL;
+    st = project_common(cfg, x, w_qkv, bias, q_out, dev_status);
+    if (st != BT_OK) return st;
+    if (n_rows <= 0) return BT_ERR_SHAPE;
+    if (n_rows > local_cap(cfg)) return BT_ERR_CAPACITY;
+    if (!local_cache_aligned(cache)) return BT_ERR_UNSUPPORTED;
+    return qkv_project(cfg, local_view(cfg, cache, layer), x, n_rows, w_qkv, bias, reset_first, reset_mask, q_out, dev_status, stream);
 }
 
 bt_status bt_selftest_bounded_wait(uint32_t* report, uint32_t* dev_status, void* stream)

@@ -97,4 +97,29 @@ cudaError_t launch_block_prefill_simple(const PrefillArgs& a, cudaStream_t strea
 bool prefill_tc_supported(const PrefillArgs& a);
 cudaError_t launch_block_prefill_tc(const PrefillArgs& a, uint32_t* dev_status, cudaStream_t stream);
 
+
+// y = W x + b on the tensor cores.  x [M][K], w [N][K] (row o = weights of output feature o), bias [N] or
+// NULL, all bf16; fp32 accumulation, bf16 results.
+//   kProjectPlain : out [M][N]
+//   kProjectQkv   : M = B * n_rows rows (sequence b, row i), N = 3 * H * hd output features ordered Q, K, V,
+//                   each (h, d): Q -> out [B][H][n_rows][hd]; K, V -> rows len_old[b] + i of `cache`
+//                   (len_old = 0 where the reset applies); a sequence without room for n_rows rows keeps
+//                   its cache.  A second launch then advances the lengths (and flags those sequences).
+enum { kProjectPlain = 0, kProjectQkv = 1 };
+struct ProjectArgs {
+    const void* x;
+    const void* w;
+    const void* bias;
+    void* out;
+    int M, N, K;
+    int mode;
+    CacheView cache;          // kProjectQkv
+    int n_rows, H, hd;        // kProjectQkv
+    int reset_first;
+    const uint8_t* reset_mask;
+    uint32_t* dev_status;
+};
+bool project_supported(const ProjectArgs& a);
+cudaError_t launch_project(const ProjectArgs& a, cudaStream_t stream);
+
 }  // namespace bt

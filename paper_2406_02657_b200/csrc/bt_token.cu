@@ -161,7 +161,8 @@ __global__ void __launch_bounds__(256, BT_TOK_MINBLOCKS) token_decode_kernel(Tok
             }
         }
     } else {
-        // general step: n_q rows (the P prefix rows at a block start), or attend-only.
+        // general step: n_q rows (the P prefix rows at a block start), or attend-only (n_q queries over rows
+        // that a projection has already cached).
         // New rows are written first; each lane later re-reads only bytes it wrote itself.
         if (active && appended && !overflow)
             for (int i = 0; i < a.n_q; ++i) {
@@ -174,7 +175,8 @@ __global__ void __launch_bounds__(256, BT_TOK_MINBLOCKS) token_decode_kernel(Tok
             unpack8(qr, qf);
 #pragma unroll
             for (int d = 0; d < 8; ++d) qf[d] *= a.scale_log2;
-            const int n = (!active || overflow) ? 0 : (appended ? len_old + i + 1 : len_old);
+            // attend only: the queries are those of the last n_q cached rows, the same causal rule counted from the end
+            const int n = (!active || overflow) ? 0 : (appended ? len_old + i + 1 : len_old - a.n_q + i + 1);
             SoftmaxState st;
             st.init();
             for (int j = 0; j < a.cap; ++j) {
@@ -199,7 +201,7 @@ __global__ void __launch_bounds__(256, BT_TOK_MINBLOCKS) token_decode_kernel(Tok
             raise_status(a.dev_status, BT_DEV_OVERFLOW);  // sequence skipped, length unchanged
         } else {
             a.len[b] = appended ? len_old + a.n_q : len_old;
-            if (!appended && len_old == 0) raise_status(a.dev_status, BT_DEV_EMPTY);
+            if (!appended && len_old < a.n_q) raise_status(a.dev_status, BT_DEV_EMPTY);  // a query with nothing to see
         }
     }
 }

@@ -87,7 +87,7 @@ def test_host_detectable_errors_return_before_launch(bt):
     assert L.bt_local_kv_reset(ref(cfg), None, 0, None, None) == bt.BT_ERR_NULL
     assert L.bt_local_kv_append(ref(cfg), ref(lc), 0, fake, fake, 6, None, None) == bt.BT_ERR_CAPACITY
     assert L.bt_token_decode_attn(ref(cfg), ref(lc), 0, fake, fake, None, 1, 0, None, fake, None, None) == bt.BT_ERR_NULL
-    assert L.bt_token_decode_attn(ref(cfg), ref(lc), 0, fake, None, None, 2, 0, None, fake, None, None) == bt.BT_ERR_SHAPE
+    assert L.bt_token_decode_attn(ref(cfg), ref(lc), 0, fake, None, None, 6, 0, None, fake, None, None) == bt.BT_ERR_CAPACITY
     assert L.bt_token_decode_attn(ref(cfg), ref(lc), 0, fake, fake, fake, 6, 0, None, fake, None, None) == bt.BT_ERR_CAPACITY
     assert L.bt_token_decode_attn(ref(cfg), ref(lc), 0, fake, fake, fake, 0, 0, None, fake, None, None) == bt.BT_ERR_SHAPE
     assert L.bt_token_decode_attn(ref(cfg), ref(lc), 0, fake, fake, fake, 1, 0, None, None, None, None) == bt.BT_ERR_NULL
@@ -95,6 +95,17 @@ def test_host_detectable_errors_return_before_launch(bt):
     assert L.bt_block_prefill_attn(ref(cfg), fake, fake, fake, 0, 8, fake, None, None) == bt.BT_ERR_SHAPE
     assert L.bt_block_prefill_attn(ref(cfg), fake, fake, fake, 16, 8, fake, None, None) == bt.BT_ERR_SHAPE
     assert L.bt_block_prefill_attn(ref(cfg), fake, None, fake, 8, 8, fake, None, None) == bt.BT_ERR_NULL
+    # projections
+    assert L.bt_prefix_project(ref(cfg), fake, None, None, fake, None, None) == bt.BT_ERR_NULL
+    assert L.bt_prefix_project(ref(bad), fake, fake, None, fake, None, None) == bt.BT_ERR_UNSUPPORTED
+    assert L.bt_block_qkv_project_append(ref(cfg), ref(bc), 0, fake, 65, fake, None, fake, None, None) == bt.BT_ERR_CAPACITY
+    assert L.bt_block_qkv_project_append(ref(cfg), ref(bc), 0, fake, 0, fake, None, fake, None, None) == bt.BT_ERR_SHAPE
+    assert L.bt_block_qkv_project_append(ref(cfg), ref(nullc), 0, fake, 1, fake, None, fake, None, None) == bt.BT_ERR_NULL
+    assert L.bt_block_qkv_project_append(ref(cfg), ref(bc), 2, fake, 1, fake, None, fake, None, None) == bt.BT_ERR_SHAPE
+    assert L.bt_local_qkv_project_append(ref(cfg), ref(lc), 0, fake, 6, fake, None, 0, None, fake, None, None) == bt.BT_ERR_CAPACITY
+    assert L.bt_local_qkv_project_append(ref(cfg), ref(lc), 0, fake, 1, None, None, 0, None, fake, None, None) == bt.BT_ERR_NULL
+    assert L.bt_local_qkv_project_append(ref(cfg), ref(lc), 0, fake, 1, fake, ctypes.c_void_p(0x1002), 0, None, fake, None, None) \
+        == bt.BT_ERR_UNSUPPORTED
     # host-driven step
     assert L.bt_block_decode_step_host(ref(cfg), ref(bc), 0, None, fake, fake, fake, fake, fake, fake, fake,
                                        None, 0, None, None) == bt.BT_ERR_NULL

@@ -43,3 +43,19 @@ def local_kv_split(kv_t):
     """local cache tensor [..., C, 2, hd] (one layer: [B,H,C,2,hd]) -> K bits, V bits [B,H,C,hd]."""
     bits = gen.torch_to_bits(kv_t)
     return np.ascontiguousarray(bits[..., 0, :]), np.ascontiguousarray(bits[..., 1, :])
+
+
+# The projections accumulate K products in fp32 on the tensor cores and round once to bf16: half a bf16
+# ulp (2^-9 relative) plus the accumulation error, which grows with sum_k |x_k w_k| (about 0.64 K for
+# N(0,1) inputs) times a few fp32 ulps - 2e-3 covers K up to 2048.
+PROJ_ATOL, PROJ_RTOL = 2e-3, 4e-3
+
+
+def assert_close_proj(gpu_bf16, ref, what=""):
+    g = to_f64(gpu_bf16).reshape(ref.shape)
+    assert np.isfinite(g).all(), f"{what}: non-finite output"
+    err = np.abs(g - ref)
+    assert (err <= ATOL + RTOL * np.abs(ref)).all(), f"{what}: max err {err.max():.3e} beyond the stated tolerance"
+    tight = PROJ_ATOL + PROJ_RTOL * np.abs(ref)
+    assert (err <= tight).all(), f"{what}: max err {err.max():.3e} beyond fp32-accumulate + bf16 rounding"
+    return err.max()
