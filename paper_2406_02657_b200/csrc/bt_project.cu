@@ -63,6 +63,18 @@ __device__ __forceinline__ bool wait(uint32_t bar, uint32_t parity, volatile int
     return false;
 }
 
+// New length of sequence b after its n rows: (reset ? 0 : len) + n when they fit, else unchanged and flagged.
+__device__ __forceinline__ void advance_len(int32_t* len, int b, int n, int cap, int reset_first, const uint8_t* reset_mask,
+                                            uint32_t* dev_status)
+{
+    const bool rst = reset_mask ? (reset_mask[b] != 0) : (reset_first != 0);
+    const int l = rst ? 0 : len[b];
+    if (l >= 0 && l + n <= cap)
+        len[b] = l + n;
+    else
+        raise_status(dev_status, BT_DEV_OVERFLOW);  // the sequence keeps its rows and its length
+}
+
 template <int BN>
 __global__ void __launch_bounds__(kThreads, 1)
 project_tc_kernel(const __grid_constant__ CUtensorMap mapX, const __grid_constant__ CUtensorMap mapW, Params p)
@@ -107,8 +119,9 @@ project_tc_kernel(const __grid_constant__ CUtensorMap mapX, const __grid_constan
     tc_fence_after();
     const uint32_t tmem = *tmem_slot;
 
+    // Programmatic dependent launch: until the kernel before this one in the stream is done, nothing here
+    // reads or writes global memory (the descriptor prefetch below touches only the kernel's own parameters).
     pdl_launch_dependents();
-    pdl_wait();  // nothing above touched global memory
 
     const int n_tiles = p.tiles_m * p.tiles_n;
     const int n_kb = (a.K + BK - 1) / BK;
@@ -117,6 +130,7 @@ project_tc_kernel(const __grid_constant__ CUtensorMap mapX, const __grid_constan
         if (lane == 0) {
             asm volatile("prefetch.tensormap [%0];" ::"l"(&mapX) : "memory");
             asm volatile("prefetch.tensormap [%0];" ::"l"(&mapW) : "memory");
+            pdl_wait();
             uint32_t it = 0;
             bool ok = true;
             for (int tile = blockIdx.x; ok && tile < n_tiles; tile += gridDim.x) {
@@ -171,6 +185,7 @@ project_tc_kernel(const __grid_constant__ CUtensorMap mapX, const __grid_constan
         const int D = a.H * a.hd;
         uint32_t t = 0;
         bool ok = true;
+        pdl_wait();
         for (int tile = blockIdx.x; tile < n_tiles; tile += gridDim.x, ++t) {
             const int tm = tile / p.tiles_n, tn = tile - tm * p.tiles_n;
             const uint32_t acc = t & 1;
@@ -220,6 +235,26 @@ project_tc_kernel(const __grid_constant__ CUtensorMap mapX, const __grid_constan
                     asm volatile("st.shared.v4.b32 [%0], {%1, %2, %3, %4};" ::"r"(dst), "r"(w.x), "r"(w.y), "r"(w.z), "r"(w.w) : "memory");
                 }
                 __syncwarp();
+                // Where the piece goes.  head_dim is a multiple of 64 and so is col0: the 64 columns lie inside one
+                // head of one of Q, K, V, so everything but the row is the same for the whole warp.
+                bf16* piece_base = reinterpret_cast<bf16*>(a.out);
+                size_t slab_elems = 0, row_elems = 0;     // element strides: per (sequence, head) slab, per row
+                int piece_h = 0, piece_d = 0;
+                bool to_cache = false;
+                if (a.mode == kProjectQkv) {
+                    const int part = col0 / D, cc = col0 - part * D;   // 0: Q, 1: K, 2: V
+                    piece_h = cc / a.hd;
+                    piece_d = cc - piece_h * a.hd;
+                    to_cache = part != 0;
+                    if (to_cache) {
+                        piece_base = reinterpret_cast<bf16*>(part == 1 ? a.cache.k : a.cache.v);
+                        slab_elems = (size_t)a.cache.slab_stride;
+                        row_elems = (size_t)a.cache.row_stride;
+                    } else {
+                        slab_elems = (size_t)a.n_rows * a.hd;
+                        row_elems = (size_t)a.hd;
+                    }
+                }
                 // out of the patch: 8 lanes take one row's 128 bytes, so every store instruction writes 4 whole lines
 #pragma unroll
                 for (int itr = 0; itr < 8; ++itr) {
@@ -233,18 +268,10 @@ project_tc_kernel(const __grid_constant__ CUtensorMap mapX, const __grid_constan
                     const int col = col0 + q8 * 8;
                     if (b < 0 || col >= a.N) continue;
                     bf16* dst = nullptr;
-                    if (a.mode == kProjectPlain) {
-                        dst = reinterpret_cast<bf16*>(a.out) + (size_t)b * a.N + col;
-                    } else {
-                        const int part = col / D, cc = col - part * D;   // 0: Q, 1: K, 2: V
-                        const int h = cc / a.hd, d = cc - h * a.hd;
-                        const size_t slab = (size_t)b * a.H + h;
-                        if (part == 0)
-                            dst = reinterpret_cast<bf16*>(a.out) + (slab * a.n_rows + i) * a.hd + d;
-                        else if (rc >= 0)
-                            dst = reinterpret_cast<bf16*>(part == 1 ? a.cache.k : a.cache.v) + slab * a.cache.slab_stride +
-                                  (size_t)rc * a.cache.row_stride + d;
-                    }
+                    if (a.mode == kProjectPlain)
+                        dst = piece_base + (size_t)b * a.N + col;
+                    else if (!to_cache || rc >= 0)   // Q row i of the sequence, or cache row rc (absent when there is no room)
+                        dst = piece_base + ((size_t)b * a.H + piece_h) * slab_elems + (size_t)(to_cache ? rc : i) * row_elems + piece_d + q8 * 8;
                     if (dst) *reinterpret_cast<uint4*>(dst) = w;
                 }
                 __syncwarp();  // the patch is free for the next piece
@@ -261,22 +288,35 @@ project_tc_kernel(const __grid_constant__ CUtensorMap mapX, const __grid_constan
         tc_fence_after();
         asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem), "r"(C::kTmemCols) : "memory");
     }
+    // With a sync word the lengths go up inside this launch: every CTA counts itself in once all of its tiles are
+    // stored (the barrier above: all epilogue warps are through), and the one that arrives last - when nobody
+    // reads the old lengths any more - advances them and puts the word back to zero.
+    if (a.mode == kProjectQkv && a.sync_word != nullptr) {
+        __shared__ int is_last;
+        if (threadIdx.x == 0) {
+            __threadfence();
+            is_last = atomicAdd(a.sync_word, 1u) == gridDim.x - 1;
+        }
+        __syncthreads();
+        if (is_last) {
+            pdl_wait();  // not every thread of the CTA has been through it yet
+            __threadfence();
+            const int B = a.M / a.n_rows;
+            for (int b = threadIdx.x; b < B; b += blockDim.x) advance_len(a.cache.len, b, a.n_rows, a.cache.cap, a.reset_first, a.reset_mask, a.dev_status);
+            if (threadIdx.x == 0) *a.sync_word = 0u;
+        }
+    }
 }
 
-// The lengths go up once every tile has read the old ones: a second, tiny launch behind the product.
+// The lengths go up once every tile has read the old ones: without a sync word, a second, tiny launch
+// behind the product.
 __global__ void project_len_advance_kernel(int32_t* len, int B, int n, int cap, int reset_first, const uint8_t* reset_mask,
                                            uint32_t* dev_status)
 {
     pdl_launch_dependents();
     pdl_wait();
     const int b = blockIdx.x * blockDim.x + threadIdx.x;
-    if (b >= B) return;
-    const bool rst = reset_mask ? (reset_mask[b] != 0) : (reset_first != 0);
-    const int l = rst ? 0 : len[b];
-    if (l >= 0 && l + n <= cap)
-        len[b] = l + n;
-    else
-        raise_status(dev_status, BT_DEV_OVERFLOW);  // the sequence keeps its rows and its length
+    if (b < B) advance_len(len, b, n, cap, reset_first, reset_mask, dev_status);
 }
 
 template <int BN>
@@ -316,7 +356,7 @@ cudaError_t launch_project(const ProjectArgs& a, cudaStream_t stream)
         e = proj::launch_bn<128>(a, dev, sms, stream);
     else
         e = proj::launch_bn<64>(a, dev, sms, stream);
-    if (e != cudaSuccess || a.mode == kProjectPlain) return e;
+    if (e != cudaSuccess || a.mode == kProjectPlain || a.sync_word != nullptr) return e;
     const int B = a.M / a.n_rows;
     return launch_pdl(proj::project_len_advance_kernel, dim3((B + 255) / 256), dim3(256), 0, stream, a.cache.len, B, a.n_rows,
                       a.cache.cap, a.reset_first, a.reset_mask, a.dev_status);
