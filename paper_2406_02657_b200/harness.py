@@ -198,10 +198,12 @@ class DenseDecodeStep:
         torch.cuda.synchronize()
         self.graph = torch.cuda.CUDAGraph()
         with torch.cuda.graph(self.graph):
-            self.rewind()
-            self.step()
+            for s in range(self.sets):
+                self.rewind()
+                self.step(s)
 
     def replay(self):
+        """`sets` steps."""
         self.graph.replay()
 
 
@@ -383,3 +385,70 @@ class GenerationRun:
         else:
             for _ in range(self.n_gen_blocks // self.ring):
                 self.graph.replay()
+
+
+class ProjectRun:
+    """The linear maps either side of the attention path over all layers, with distinct weights per layer:
+    kind "qkv_token" - one token step of the token decoder (section 2.4): x [B,1,D] -> q, K and V rows into
+    the local cache (reset at every launch so that a step can be repeated); kind "qkv_block" - one block
+    step of the block decoder (section 2.3): x [B,1,D] -> q, K and V rows appended to the block cache (the
+    lengths are put back before every step); kind "prefix" - context embedding [B,D] -> P prefix embeddings.
+    ``sets`` independent copies of the per-layer tensors are used round-robin, `sets` steps per graph replay,
+    so that a replay's working set can be made larger than the L2 cache."""
+
+    def __init__(self, w, kind, device="cuda", fill=None, sets=1):
+        self.w, self.kind, self.sets = w, kind, sets
+        B, H, hd, P = w.batch, w.heads, w.head_dim, w.prefix_len
+        L = w.n_layers * sets   # tensors are [sets * layers, ...]; set s uses rows s*layers .. (s+1)*layers-1
+        D = H * hd
+        self.cfg = bt.make_config(B, H, hd, w.block_len, P, max(1, w.max_blocks), w.n_layers)
+        mk = fill if fill is not None else (lambda tid, sh: torch.zeros(sh, dtype=torch.bfloat16, device=device))
+        self.status = torch.zeros(1, dtype=torch.int32, device=device)
+        self.sync = torch.zeros(1, dtype=torch.int32, device=device)
+        if kind == "prefix":
+            self.x, self.wt, self.bias = mk(40, (L, B, D)), mk(41, (L, P * D, D)), mk(42, (L, P * D))
+            self.out = torch.empty((L, B, P, D), dtype=torch.bfloat16, device=device)
+            self.M, self.N, self.K = B, P * D, D
+        else:
+            self.x, self.wt, self.bias = mk(43, (L, B, 1, D)), mk(44, (L, 3 * D, D)), mk(45, (L, 3 * D))
+            self.out = torch.empty((L, B, H, 1, hd), dtype=torch.bfloat16, device=device)
+            self.M, self.N, self.K = B, 3 * D, D
+            L = w.n_layers
+            if kind == "qkv_token":
+                self.cache = bt.LocalCache(self.cfg, device)
+            else:
+                self.cache = bt.BlockCache(self.cfg, device)
+                self.len0 = torch.full((L, B), w.ctx_blocks - 1, dtype=torch.int32, device=device)
+                self.cache.len.copy_(self.len0)
+        self.launches_per_step = w.n_layers
+        self.graph = None
+
+    def step(self, s=0):
+        for l in range(self.w.n_layers):
+            i = s * self.w.n_layers + l
+            if self.kind == "prefix":
+                bt.bt_prefix_project(self.cfg, self.x[i], self.wt[i], self.bias[i], self.out[i], dev_status=self.status)
+            elif self.kind == "qkv_token":
+                bt.bt_local_qkv_project_append(self.cfg, self.cache, l, self.x[i], self.wt[i], self.bias[i], self.out[i],
+                                               reset_first=True, sync_word=self.sync, dev_status=self.status)
+            else:
+                bt.bt_block_qkv_project_append(self.cfg, self.cache, l, self.x[i], self.wt[i], self.bias[i], self.out[i],
+                                               sync_word=self.sync, dev_status=self.status)
+
+    def rewind(self):
+        if self.kind == "qkv_block":
+            self.cache.len.copy_(self.len0, non_blocking=True)
+
+    def capture(self):
+        self.rewind()
+        self.step()
+        torch.cuda.synchronize()
+        self.graph = torch.cuda.CUDAGraph()
+        with torch.cuda.graph(self.graph):
+            for s in range(self.sets):
+                self.rewind()
+                self.step(s)
+
+    def replay(self):
+        """`sets` steps."""
+        self.graph.replay()

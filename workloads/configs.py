@@ -63,6 +63,16 @@ BLOCK_PREFILL_8K = Workload("block_prefill_8k", batch=8, heads=16, head_dim=128,
                             n_layers=12, max_blocks=2048, prompt_blocks=2048, prompt_tokens=8192, seed=1014)
 
 
+# the linear maps either side of the path, at the shapes of configs 3 and 2: one token step of the token decoder
+# (4096 rows), one block step of the block decoder (256 rows), model dim 1024, distinct weights per layer
+QKV_PROJECT_TOKEN = Workload("qkv_project_token", batch=4096, heads=16, head_dim=64, block_len=4, prefix_len=1,
+                             n_layers=12, max_blocks=1, seed=1033)
+QKV_PROJECT_BLOCK = Workload("qkv_project_block", batch=256, heads=16, head_dim=64, block_len=4, prefix_len=1,
+                             n_layers=12, max_blocks=512, ctx_blocks=512, seed=1032)
+PREFIX_PROJECT = Workload("prefix_project", batch=4096, heads=16, head_dim=64, block_len=4, prefix_len=2,
+                          n_layers=12, max_blocks=1, seed=1034)
+
+
 def sweep(block_len: int) -> Workload:
     """config 5: decode-heavy generation (128-token prompt, 2048 generated) at one block length."""
     prompt, gen = 128, 2048
@@ -77,4 +87,5 @@ def scaled(w: Workload, **kw) -> Workload:
     return replace(w, **kw)
 
 
-BY_NAME = {w.name: w for w in (TINY, BLOCK_DECODE, BLOCK_DECODE_16K, DENSE_DECODE, TOKEN_DECODE, BLOCK_PREFILL, BLOCK_PREFILL_8K)}
+BY_NAME = {w.name: w for w in (TINY, BLOCK_DECODE, BLOCK_DECODE_16K, DENSE_DECODE, TOKEN_DECODE, BLOCK_PREFILL, BLOCK_PREFILL_8K,
+                               QKV_PROJECT_TOKEN, QKV_PROJECT_BLOCK, PREFIX_PROJECT)}

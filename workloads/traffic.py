@@ -59,3 +59,13 @@ def generation_bytes(B: int, H: int, hd: int, n_layers: int, block_len: int, pro
     token = n_layers * G * sum(token_decode_layer_bytes(B, H, hd, j) for j in range(block_len))
     block = n_layers * sum(block_decode_layer_bytes(B, H, hd, T + g + 1, True) for g in range(G))
     return {"prefill": prefill, "token": token, "block": block, "total": prefill + token + block}
+
+
+def linear_flops(M: int, N: int, K: int) -> int:
+    """y = W x + b over M rows: one multiply-add per (row, output feature, input feature)."""
+    return 2 * M * N * K
+
+
+def linear_bytes(M: int, N: int, K: int) -> int:
+    """x [M,K] and W [N,K] read once, bias [N] read once, y [M,N] written once (wherever its parts go)."""
+    return (M * K + N * K + N + M * N) * BF16
