@@ -237,7 +237,10 @@ NCU_TRAFFIC_BYTES = {
     # reads equal the algorithmic reads; the 25.2 MB written per launch mostly reach DRAM after the launch and
     # are counted at their algorithmic size
     ("token_decode", 1): 75.5e6,
-    ("block_prefill", 1): None,        # the kernel changed since the last capture
+    ("block_prefill", 1): 220.4e6,     # 110.2 MB captured at batch 16 (reads exact; 9.4 of 33.5 MB of writes reach DRAM inside the launch)
+    # reads are x and W exactly once (14.7 MB); the 25.2 MB of q, K, V rows written stay in L2 until after the launch
+    # and are counted at their algorithmic size
+    ("qkv_project_token", 1): 39.9e6,
 }
 
 
@@ -441,7 +444,8 @@ def measure(name, w, args, env, primary):
         assert run.status.item() == 0 and run.sync.item() == 0
         alg = traffic.linear_bytes(run.M, run.N, run.K)
         fl = traffic.linear_flops(run.M, run.N, run.K)
-        roof = hbm_roofline(pk, "project_tc_kernel", alg, ms / w.n_layers, w.n_layers * alg, ms, None)
+        roof = hbm_roofline(pk, "project_tc_kernel", alg, ms / w.n_layers, w.n_layers * alg, ms,
+                            NCU_TRAFFIC_BYTES.get((name, 1)) if w.batch == 4096 else None)
         add_tensor_roofline(roof, pk, fl, alg, ms / w.n_layers, in_long_step=False)
         launches = run.launches_per_step * steps
         if not args.no_cpu_baseline:
@@ -485,7 +489,7 @@ def measure(name, w, args, env, primary):
 # what the default run measures after its primary line: (workload, prefix length, block length, steps, warm-up)
 SECONDARY = [
     # step counts sized for about half a second of timed work each, so that the clock sampler sees the region
-    ("token_decode", 1, 0, 400, 3), ("token_decode", 2, 0, 300, 3), ("block_prefill", 0, 0, 600, 3), ("block_prefill_8k", 0, 0, 250, 3),
+    ("token_decode", 1, 0, 400, 3), ("token_decode", 2, 0, 300, 3), ("token_decode", 8, 0, 150, 3), ("block_prefill", 0, 0, 600, 3), ("block_prefill_8k", 0, 0, 250, 3),
     ("qkv_project_token", 0, 0, 1200, 3), ("qkv_project_block", 0, 0, 2000, 3), ("prefix_project", 0, 0, 2000, 3),
     ("sweep", 0, 4, 2, 1), ("sweep", 0, 8, 2, 1),
 ]

@@ -449,7 +449,7 @@ cudaError_t launch_token_decode(const TokenArgs& a, cudaStream_t stream)
 {
     const int lpr = a.hd / 8;
     const int tps = a.H * lpr;  // threads per sequence (validated <= 256 by the caller)
-    if (a.n_q == 1 && a.k_new != nullptr && a.cap - 1 <= 8) {
+    if (a.n_q == 1 && a.k_new != nullptr && a.cap - 1 <= 12) {
         // hot path: persistent pipelined kernel; deeper pipeline when the slots are small
         int spc_p = kTokThreads / tps;
         if (spc_p > a.B) spc_p = a.B;
@@ -459,6 +459,16 @@ cudaError_t launch_token_decode(const TokenArgs& a, cudaStream_t stream)
         if (a.cap - 1 <= 5)  // e.g. L_B = 4 with the paper's main prefix length P = 2: still two CTAs per SM
             return a.hd == 64 ? launch_pipelined<64, 1, 5, 2>(a, spc_p, tps, stream)
                               : launch_pipelined<128, 1, 5, 2>(a, spc_p, tps, stream);
+        if (a.cap - 1 > 8)  // the longest prefixes of the prefix-length ablation (P = 8 with L_B up to 5): 9 to 12 cached rows
+            return a.hd == 64 ? launch_pipelined<64, 1, 12, 1>(a, spc_p, tps, stream)
+                              : launch_pipelined<128, 1, 12, 1>(a, spc_p, tps, stream);
+        // Deep local caches (6 to 8 cached rows).  A batch small enough for one wave of two CTAs per SM runs
+        // without a look-ahead stage (each CTA has a single group, so there is nothing to look ahead to, and
+        // the halved slots let all groups be resident at once); larger ones keep one group in flight per SM.
+        int dev = 0, sms = 0;
+        if (current_device(&dev, &sms) == cudaSuccess && (a.B + spc_p - 1) / spc_p <= 2 * sms)
+            return a.hd == 64 ? launch_pipelined<64, 0, 8, 2>(a, spc_p, tps, stream)
+                              : launch_pipelined<128, 0, 8, 2>(a, spc_p, tps, stream);
         return a.hd == 64 ? launch_pipelined<64, 1, 8, 1>(a, spc_p, tps, stream)
                           : launch_pipelined<128, 1, 8, 1>(a, spc_p, tps, stream);
     }
