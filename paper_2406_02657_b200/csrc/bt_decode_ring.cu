@@ -30,7 +30,7 @@ namespace ring {
 #define BT_DEC_WARPS 8
 #endif
 #ifndef BT_DEC_MAX_WARPS
-#define BT_DEC_MAX_WARPS 9
+#define BT_DEC_MAX_WARPS 12
 #endif
 #ifndef BT_DEC_STAGES
 #define BT_DEC_STAGES 3
@@ -41,7 +41,9 @@ namespace ring {
 // Warps per CTA are chosen per launch (kMinWarps..kMaxWarps, kWarps unless another count leaves fewer
 // warps idle in the last round of items): every warp has its own ring, so the kernel only needs the count.
 constexpr int kWarps = BT_DEC_WARPS;
-constexpr int kMinWarps = 6, kMaxWarps = BT_DEC_MAX_WARPS;
+constexpr int kMinWarps = 6, kMaxWarps = BT_DEC_MAX_WARPS;   // the register budget allows twelve (two-stage rings only)
+constexpr int kMaxWarpsLong = 9;      // most warps considered when the rows may be many
+constexpr int kShortCacheRows = 320;  // capacity up to which an item is short enough for twelve warps to pay
 constexpr int kMaxThreads = kMaxWarps * 32;
 // Ring depth, chosen per launch: two stages when at least three warps in four have an item (with the
 // memory system saturated by many rings, less in flight per warp runs faster: 82.4 vs 84.2 us at 4096
@@ -86,12 +88,53 @@ struct Work {
     int bh, sp, b, n, r0, c1;
     bool new_row, overflow;
 };
-__device__ __forceinline__ Work decode_work(int item, const DecodeArgs& a)
+// Position of a warp in the line of items: item = bh * splits + sp, bh = b * H + h.  A warp walks the line with a
+// fixed stride, so the parts are carried forward by additions (the divisions happen once, in Step): with caches of
+// a few dozen rows an item is a thousand instructions, and integer divisions were a sixth of them.
+struct Cursor {
+    int item, bh, sp, b, h;
+};
+struct Step {   // stride split into its parts
+    int items, bh, sp, b, h;
+};
+__device__ __forceinline__ Cursor cursor_at(int item, const DecodeArgs& a)
+{
+    Cursor c;
+    c.item = item;
+    c.bh = item / a.splits;
+    c.sp = item - c.bh * a.splits;
+    c.b = c.bh / a.H;
+    c.h = c.bh - c.b * a.H;
+    return c;
+}
+__device__ __forceinline__ Step step_of(int stride, const DecodeArgs& a)
+{
+    Step s;
+    s.items = stride;
+    s.bh = stride / a.splits;
+    s.sp = stride - s.bh * a.splits;
+    s.b = s.bh / a.H;
+    s.h = s.bh - s.b * a.H;
+    return s;
+}
+__device__ __forceinline__ void advance(Cursor& c, const Step& s, const DecodeArgs& a)
+{
+    c.item += s.items;
+    c.sp += s.sp;
+    const int carry_sp = c.sp >= a.splits ? 1 : 0;
+    c.sp -= carry_sp ? a.splits : 0;
+    c.bh += s.bh + carry_sp;
+    c.h += s.h + carry_sp;              // < 2 H
+    const int carry_h = c.h >= a.H ? 1 : 0;
+    c.h -= carry_h ? a.H : 0;
+    c.b += s.b + carry_h;
+}
+__device__ __forceinline__ Work decode_work(const Cursor& c, const DecodeArgs& a)
 {
     Work w;
-    w.bh = item / a.splits;
-    w.sp = item - w.bh * a.splits;
-    w.b = w.bh / a.H;
+    w.bh = c.bh;
+    w.sp = c.sp;
+    w.b = c.b;
     int n = a.len[w.b];
     n = n < 0 ? 0 : (n > a.n_max ? a.n_max : n);
     const bool append = a.k_new != nullptr && n < a.n_max;  // a full cache takes no row: flagged, attended as it is
@@ -159,22 +202,25 @@ __global__ void __launch_bounds__(kMaxThreads, 1) block_decode_ring_kernel(Decod
     pdl_wait();  // nothing above wrote global memory, or used a value read from it for more than a prefetch hint
 
     // ---- producer cursor (kept by every lane, acted on by lane 0): next chunk to request
-    int p_item = first, p_c = 0, p_nchunks = 0;
+    const Step step = step_of(stride, a);
+    Cursor pc = cursor_at(first < n_items ? first : 0, a);
+    pc.item = first;
+    int p_c = 0, p_nchunks = 0;
     Work pw = {};
     auto p_seek = [&]() {  // move to the next item that has rows
-        while (p_item < n_items) {
-            pw = decode_work(p_item, a);
+        while (pc.item < n_items) {
+            pw = decode_work(pc, a);
             p_nchunks = (pw.c1 - pw.r0 + ROWS - 1) / ROWS;
             if (p_nchunks > 0) {
                 p_c = 0;
                 return;
             }
-            p_item += stride;
+            advance(pc, step, a);
         }
     };
     uint32_t issued = 0, consumed = 0;
     auto issue_one = [&]() {
-        if (p_item >= n_items) return;
+        if (pc.item >= n_items) return;
         const int row = pw.r0 + p_c * ROWS;
         const uint32_t bytes = (uint32_t)min(ROWS, pw.c1 - row) * G::ROW_BYTES;
         const uint32_t st = issued % kStages;
@@ -187,7 +233,7 @@ __global__ void __launch_bounds__(kMaxThreads, 1) block_decode_ring_kernel(Decod
         }
         ++issued;
         if (++p_c == p_nchunks) {
-            p_item += stride;
+            advance(pc, step, a);
             p_seek();
         }
     };
@@ -198,9 +244,34 @@ __global__ void __launch_bounds__(kMaxThreads, 1) block_decode_ring_kernel(Decod
     bool alive = true;
     const bf16* Qall = reinterpret_cast<const bf16*>(a.q);
     uint4 q_next = make_uint4(0, 0, 0, 0);  // the query of the next item is fetched an item ahead
-    if (first < n_items) q_next = ld_plain(Qall + (size_t)(first / a.splits) * HD + sub * 8);
-    for (int item = first; alive && item < n_items; item += stride) {
-        const Work w = decode_work(item, a);
+    // ... and so is the row to append (whichever item of the (sequence, head) turns out to own it: the loads are
+    // speculative and cost 2 x 16 bytes per lane group).  With caches of a few dozen rows an item is over sooner
+    // than a round trip to DRAM, so nothing an item needs may be requested inside it.
+    uint4 kn_next = make_uint4(0, 0, 0, 0), vn_next = kn_next;
+    Cursor cc = cursor_at(first < n_items ? first : 0, a);   // this item
+    cc.item = first;
+    Cursor cn = cc;                                          // the item after it
+    advance(cn, step, a);
+    if (first < n_items) {
+        q_next = ld_plain(Qall + (size_t)cc.bh * HD + sub * 8);
+        if (a.k_new != nullptr) {
+            kn_next = ld_plain(reinterpret_cast<const bf16*>(a.k_new) + (size_t)cc.bh * HD + sub * 8);
+            vn_next = ld_plain(reinterpret_cast<const bf16*>(a.v_new) + (size_t)cc.bh * HD + sub * 8);
+        }
+    }
+    // The length update of an item is settled one item later, for the same reason: the count it depends on comes
+    // back from L2.  (lane 0 only)
+    int pend_arrival = -1, pend_b = 0, pend_n = 0;
+    bool pend_overflow = false;
+    auto settle = [&]() {
+        if (pend_arrival == a.H * a.splits - 1) {
+            // that item was the last of its sequence to read the old length: raise it
+            if (!pend_overflow) a.len[pend_b] = pend_n;
+            a.counters[(size_t)a.B * a.H + pend_b] = 0;
+        }
+    };
+    for (; alive && cc.item < n_items; cc = cn, advance(cn, step, a)) {
+        const Work w = decode_work(cc, a);
         // Fused append: the sequence's length goes up once all of its H * splits items have read the old
         // one.  An item counts itself in as soon as its own read has returned (the increment is computed
         // from the value read, so the count cannot be issued before that) and looks at the result only
@@ -215,16 +286,17 @@ __global__ void __launch_bounds__(kMaxThreads, 1) block_decode_ring_kernel(Decod
         float qf[8];
         {
             const uint4 qr = q_next;
-            if (item + stride < n_items) q_next = ld_plain(Qall + (size_t)((item + stride) / a.splits) * HD + sub * 8);
+            if (cn.item < n_items) q_next = ld_plain(Qall + (size_t)cn.bh * HD + sub * 8);
             unpack8(qr, qf);
 #pragma unroll
             for (int i = 0; i < 8; ++i) qf[i] *= a.scale_log2;
         }
-        // the appended row, when this item owns it: fetched now, used after the cached rows
-        uint4 kn = make_uint4(0, 0, 0, 0), vn = kn;
-        if (w.new_row) {
-            kn = ld_plain(reinterpret_cast<const bf16*>(a.k_new) + (size_t)w.bh * HD + sub * 8);
-            vn = ld_plain(reinterpret_cast<const bf16*>(a.v_new) + (size_t)w.bh * HD + sub * 8);
+        // the row to append (used only if this item owns it), fetched an item ago; the next item's is requested now
+        const uint4 kn = kn_next, vn = vn_next;
+        if (a.k_new != nullptr && cn.item < n_items) {
+            const size_t nb = (size_t)cn.bh * HD + sub * 8;
+            kn_next = ld_plain(reinterpret_cast<const bf16*>(a.k_new) + nb);
+            vn_next = ld_plain(reinterpret_cast<const bf16*>(a.v_new) + nb);
         }
         SoftmaxState st;
         st.init();
@@ -263,6 +335,7 @@ __global__ void __launch_bounds__(kMaxThreads, 1) block_decode_ring_kernel(Decod
                 }
             } else {  // ragged tail: rows past the range were not copied and count as absent
                 const uint4 zero = make_uint4(0, 0, 0, 0);
+                const int ngroups = (nvalid + RPW - 1) / RPW;   // groups of RPW rows that hold any row at all (warp-uniform)
 #pragma unroll
                 for (int u = 0; u < kUnroll; ++u) {
                     const bool valid = u * RPW + rg < nvalid;
@@ -272,10 +345,30 @@ __global__ void __launch_bounds__(kMaxThreads, 1) block_decode_ring_kernel(Decod
                 refill();
 #pragma unroll
                 for (int u = 0; u < kUnroll; ++u) {
-                    const float d = row_sum<LPR>(dot8(qf, kr[u]));
-                    s[u] = (u * RPW + rg < nvalid) ? d : kNegInf;
-                    mt = fmaxf(mt, s[u]);
+                    s[u] = kNegInf;
+                    if (u < ngroups) {
+                        const float d = row_sum<LPR>(dot8(qf, kr[u]));
+                        s[u] = (u * RPW + rg < nvalid) ? d : kNegInf;
+                        mt = fmaxf(mt, s[u]);
+                    }
                 }
+                if (mt != kNegInf) {  // uniform within the LPR lanes of a row group
+                    const float mn = fmaxf(st.m, mt);
+                    const float cf = ex2(st.m - mn);
+                    st.l *= cf;
+#pragma unroll
+                    for (int i = 0; i < 8; ++i) st.acc[i] *= cf;
+#pragma unroll
+                    for (int u = 0; u < kUnroll; ++u) {
+                        if (u < ngroups) {
+                            const float p = ex2(s[u] - mn);   // 0 for the absent rows of the last group
+                            st.l += p;
+                            fma8(st.acc, p, vr[u]);
+                        }
+                    }
+                    st.m = mn;
+                }
+                continue;
             }
             if (mt != kNegInf) {  // uniform within the LPR lanes of a row group
                 const float mn = fmaxf(st.m, mt);
@@ -362,16 +455,17 @@ __global__ void __launch_bounds__(kMaxThreads, 1) block_decode_ring_kernel(Decod
                 if (lane == 0) a.counters[w.bh] = 0;
             }
         }
-        if (w.sp == 0 && (w.bh % a.H) == 0 && lane == 0) {
+        if (w.sp == 0 && cc.h == 0 && lane == 0) {
             if (w.n == 0) raise_status(a.dev_status, BT_DEV_EMPTY);
             if (w.overflow) raise_status(a.dev_status, BT_DEV_OVERFLOW);
         }
-        if (seq_arrival == a.H * a.splits - 1) {
-            // this item was the last of its sequence to read the old length (lane 0 only): raise it
-            if (!w.overflow) a.len[w.b] = w.n;
-            a.counters[(size_t)a.B * a.H + w.b] = 0;
-        }
+        settle();   // the item before this one: its count has long come back
+        pend_arrival = seq_arrival;
+        pend_b = w.b;
+        pend_n = w.n;
+        pend_overflow = w.overflow;
     }
+    settle();
     if (!alive) {
         // a copy never completed: report it, give the copies still in flight one more bounded wait so
         // that none lands in shared memory after the CTA is gone, and leave
@@ -385,7 +479,7 @@ template <int HD, int STAGES>
 static cudaError_t launch_st(const DecodeArgs& a, long long grid, int warps, int dev, cudaStream_t stream)
 {
     static PerDeviceOnce limit_raised;
-    cudaError_t e = raise_smem_limit_once(limit_raised, dev, block_decode_ring_kernel<HD, STAGES>, smem_bytes<HD>(kMaxWarps, STAGES));
+    cudaError_t e = raise_smem_limit_once(limit_raised, dev, block_decode_ring_kernel<HD, STAGES>, smem_bytes<HD>(STAGES == 2 ? kMaxWarps : kMaxWarpsLong, STAGES));
     if (e != cudaSuccess) return e;
     return launch_pdl(block_decode_ring_kernel<HD, STAGES>, dim3((unsigned)grid), dim3(warps * 32),
                       (size_t)smem_bytes<HD>(warps, STAGES), stream, a);
@@ -406,7 +500,7 @@ static cudaError_t launch_t(const DecodeArgs& a, cudaStream_t stream)
     // with the fullest last round (4096 items on 148 SMs: 7 warps run 3.95 -> 4 rounds, 8 warps 3.46 -> 4).
     int warps = kWarps;
     double best = 0.0;
-    for (int w = kMaxWarps; w >= kMinWarps; --w) {
+    for (int w = kMaxWarpsLong; w >= kMinWarps; --w) {
         const long long slots = grid * w, rounds = (items + slots - 1) / slots;
         const double fill = (double)items / (double)(rounds * slots) + (w == kWarps ? 1e-9 : 0.0);  // ties go to kWarps
         if (fill > best) {
@@ -414,7 +508,11 @@ static cudaError_t launch_t(const DecodeArgs& a, cudaStream_t stream)
             warps = w;
         }
     }
-    const bool shallow = items * 4 >= grid * warps * 3;   // (nearly) every warp has an item: the shallow ring
+    // Short caches (the capacity bounds the rows): an item is then about a thousand instructions whatever its rows,
+    // and what limits the launch is how many warps an SM has to interleave - twelve when all of them get items
+    // (17.7 vs 21.6 us at 8192 items of 17 rows; at 272 rows the same, at 512 rows eight warps win).
+    if (a.n_max <= kShortCacheRows && items >= grid * kMaxWarps) warps = kMaxWarps;
+    const bool shallow = items * 4 >= grid * warps * 3 || warps > kMaxWarpsLong;   // (nearly) every warp has an item: the shallow ring
     return shallow ? launch_st<HD, 2>(a, grid, warps, dev, stream) : launch_st<HD, kDeepStages>(a, grid, warps, dev, stream);
 }
 

@@ -108,58 +108,6 @@ __global__ void __launch_bounds__(256, BT_TOK_MINBLOCKS) token_decode_kernel(Tok
             for (int i = 0; i < 8; ++i) o[i] = st.acc[i] * inv;
             *reinterpret_cast<uint4*>(op) = pack8(o);
         }
-    } else if (appended && a.reset_first && a.reset_mask == nullptr && a.n_q <= 4) {
-        // block start (section 2.4): every sequence is reset and the P prefix rows arrive together.  There
-        // is nothing cached to read: all 3 P rows are requested at once and stay in registers, query i
-        // attends to the new rows 0..i.
-        constexpr int kMaxQ = 4;
-        uint4 qn[kMaxQ], kn[kMaxQ], vn[kMaxQ];
-#pragma unroll
-        for (int i = 0; i < kMaxQ; ++i) {
-            const bool v = active && i < a.n_q;
-            qn[i] = v ? ld_stream(qp + (size_t)i * HD) : make_uint4(0, 0, 0, 0);
-            kn[i] = v ? ld_stream(kp + (size_t)i * HD) : make_uint4(0, 0, 0, 0);
-            vn[i] = v ? ld_stream(vp + (size_t)i * HD) : make_uint4(0, 0, 0, 0);
-        }
-        const bool write = active && !overflow;  // overflow here means n_q > capacity: refused on the host already
-#pragma unroll
-        for (int i = 0; i < kMaxQ; ++i) {
-            if (i < a.n_q) {  // uniform
-                float qf[8];
-                unpack8(qn[i], qf);
-#pragma unroll
-                for (int d = 0; d < 8; ++d) qf[d] *= a.scale_log2;
-                float sc[kMaxQ];
-                float mx = kNegInf;
-#pragma unroll
-                for (int j = 0; j < kMaxQ; ++j) {
-                    if (j <= i) {
-                        sc[j] = row_sum<LPR>(dot8(qf, kn[j]));
-                        mx = fmaxf(mx, sc[j]);
-                    }
-                }
-                float l = 0.f, acc[8] = {0.f, 0.f, 0.f, 0.f, 0.f, 0.f, 0.f, 0.f};
-#pragma unroll
-                for (int j = 0; j < kMaxQ; ++j) {
-                    if (j <= i) {
-                        const float pj = ex2(sc[j] - mx);
-                        l += pj;
-                        fma8(acc, pj, vn[j]);
-                    }
-                }
-                if (active) {
-                    float o[8];
-                    const float inv = write ? 1.f / l : 0.f;
-#pragma unroll
-                    for (int d = 0; d < 8; ++d) o[d] = acc[d] * inv;
-                    *reinterpret_cast<uint4*>(op + (size_t)i * HD) = pack8(o);
-                }
-                if (write) {
-                    *reinterpret_cast<uint4*>(cache + (size_t)i * 2 * HD) = kn[i];
-                    *reinterpret_cast<uint4*>(cache + (size_t)i * 2 * HD + HD) = vn[i];
-                }
-            }
-        }
     } else {
         // general step: n_q rows (the P prefix rows at a block start), or attend-only (n_q queries over rows
         // that a projection has already cached).
@@ -204,6 +152,75 @@ __global__ void __launch_bounds__(256, BT_TOK_MINBLOCKS) token_decode_kernel(Tok
             if (!appended && len_old < a.n_q) raise_status(a.dev_status, BT_DEV_EMPTY);  // a query with nothing to see
         }
     }
+}
+
+// Block start (section 2.4): every sequence is reset and its P prefix rows arrive together, n_q = P <= kMaxQ.
+// There is nothing cached to read: all 3 P rows are requested at once and stay in registers, query i attends
+// to the new rows 0..i, the rows go to cache rows 0..P-1 and the length becomes P.  Same thread layout as the
+// general kernel (hd/8 lanes per (sequence, head), whole sequences per CTA).
+template <int HD, int kMaxQ>
+__global__ void __launch_bounds__(256) token_block_start_kernel(TokenArgs a, int seqs_per_cta, int threads_per_seq)
+{
+    constexpr int LPR = RowGeo<HD>::LPR;
+    const int tid = threadIdx.x;
+    const int sic = tid / threads_per_seq;
+    const int within = tid - sic * threads_per_seq;
+    const int h = within / LPR, sub = within % LPR;
+    const int b = blockIdx.x * seqs_per_cta + sic;
+    const bool active = sic < seqs_per_cta && b < a.B;
+    pdl_launch_dependents();
+    pdl_wait();
+    const size_t slab = active ? (size_t)b * a.H + h : 0;
+    bf16* cache = reinterpret_cast<bf16*>(a.kv) + slab * a.cap * 2 * HD + sub * 8;
+    const bf16* qp = reinterpret_cast<const bf16*>(a.q) + slab * a.n_q * HD + sub * 8;
+    const bf16* kp = reinterpret_cast<const bf16*>(a.k_new) + slab * a.n_q * HD + sub * 8;
+    const bf16* vp = reinterpret_cast<const bf16*>(a.v_new) + slab * a.n_q * HD + sub * 8;
+    bf16* op = reinterpret_cast<bf16*>(a.out) + slab * a.n_q * HD + sub * 8;
+    uint4 qn[kMaxQ], kn[kMaxQ], vn[kMaxQ];
+#pragma unroll
+    for (int i = 0; i < kMaxQ; ++i) {
+        const bool v = active && i < a.n_q;
+        qn[i] = v ? ld_stream(qp + (size_t)i * HD) : make_uint4(0, 0, 0, 0);
+        kn[i] = v ? ld_stream(kp + (size_t)i * HD) : make_uint4(0, 0, 0, 0);
+        vn[i] = v ? ld_stream(vp + (size_t)i * HD) : make_uint4(0, 0, 0, 0);
+    }
+#pragma unroll
+    for (int i = 0; i < kMaxQ; ++i) {
+        if (i < a.n_q) {  // uniform
+            float qf[8];
+            unpack8(qn[i], qf);
+#pragma unroll
+            for (int d = 0; d < 8; ++d) qf[d] *= a.scale_log2;
+            float sc[kMaxQ];
+            float mx = kNegInf;
+#pragma unroll
+            for (int j = 0; j < kMaxQ; ++j) {
+                if (j <= i) {
+                    sc[j] = row_sum<LPR>(dot8(qf, kn[j]));
+                    mx = fmaxf(mx, sc[j]);
+                }
+            }
+            float l = 0.f, acc[8] = {0.f, 0.f, 0.f, 0.f, 0.f, 0.f, 0.f, 0.f};
+#pragma unroll
+            for (int j = 0; j < kMaxQ; ++j) {
+                if (j <= i) {
+                    const float pj = ex2(sc[j] - mx);
+                    l += pj;
+                    fma8(acc, pj, vn[j]);
+                }
+            }
+            if (active) {
+                float o[8];
+                const float inv = 1.f / l;
+#pragma unroll
+                for (int d = 0; d < 8; ++d) o[d] = acc[d] * inv;
+                *reinterpret_cast<uint4*>(op + (size_t)i * HD) = pack8(o);
+                *reinterpret_cast<uint4*>(cache + (size_t)i * 2 * HD) = kn[i];
+                *reinterpret_cast<uint4*>(cache + (size_t)i * 2 * HD + HD) = vn[i];
+            }
+        }
+    }
+    if (active && within == 0) a.len[b] = a.n_q;  // nobody reads the old length here: the reset drops it
 }
 
 // ---------------------------------------------------------------------------------------
@@ -477,6 +494,14 @@ cudaError_t launch_token_decode(const TokenArgs& a, cudaStream_t stream)
     if (spc > a.B) spc = a.B;
     const int threads = ((spc * tps + 31) / 32) * 32;
     const int grid = (a.B + spc - 1) / spc;
+    if (a.k_new != nullptr && a.reset_first && a.reset_mask == nullptr && a.n_q <= 8 && a.n_q <= a.cap) {
+        // block start: the register-resident kernel (rows kept for up to 4 or up to 8 prefix rows)
+        if (a.n_q <= 4)
+            return a.hd == 64 ? launch_pdl(token_block_start_kernel<64, 4>, dim3(grid), dim3(threads), 0, stream, a, spc, tps)
+                              : launch_pdl(token_block_start_kernel<128, 4>, dim3(grid), dim3(threads), 0, stream, a, spc, tps);
+        return a.hd == 64 ? launch_pdl(token_block_start_kernel<64, 8>, dim3(grid), dim3(threads), 0, stream, a, spc, tps)
+                          : launch_pdl(token_block_start_kernel<128, 8>, dim3(grid), dim3(threads), 0, stream, a, spc, tps);
+    }
     return a.hd == 64 ? launch_pdl(token_decode_kernel<64>, dim3(grid), dim3(threads), 0, stream, a, spc, tps)
                       : launch_pdl(token_decode_kernel<128>, dim3(grid), dim3(threads), 0, stream, a, spc, tps);
 }
