@@ -18,6 +18,14 @@
 //                     tile's products
 // BN (64, 128 or 256 output features per tile) is chosen per launch so that there are enough tiles
 // for every SM.  Every wait is bounded in wall time and raises BT_DEV_TIMEOUT when it runs out.
+//
+// Large products run the same kernel on pairs of CTAs (kCtas = 2, a cluster of two SMs, tcgen05 cta_group::2):
+// a pair owns a 256 x BN tile, each CTA loads its own 128 rows of x and only HALF of the W tile (its BN/2
+// output features) with plain TMA loads - no multicast - that report to the leader CTA's barrier; the leader's
+// one MMA thread issues 256 x BN x 16 instructions that read both halves of W from the two CTAs' shared
+// memory and accumulate each CTA's 128 rows in that CTA's tensor memory; commits are multicast to both CTAs'
+// barriers; each CTA drains its own accumulator and reports to the leader.  Per CTA this moves a third less
+// operand data from L2 into shared memory for the same products.
 #include <cuda.h>
 
 #include "bt_common.cuh"
@@ -41,11 +49,13 @@ constexpr uint32_t kSpinLimit = 1u << 26;
 constexpr uint64_t kWaitLimitNs = 1000000000ull;  // 1 s: far beyond any legitimate wait
 constexpr uint32_t kPatchBytes = 32 * 128;         // per epilogue warp: 32 rows x 64 bf16
 
-template <int BN>
+constexpr uint32_t kPeerBitMask = 0xFEFFFFFFu;   // clears the bit that tells the two CTAs of a pair apart in a shared::cluster address
+
+template <int BN, int kCtas>
 struct Cfg {
-    static constexpr uint32_t kBBytes = BN * BK * 2;
+    static constexpr uint32_t kBBytes = (BN / kCtas) * BK * 2;   // a CTA of a pair holds half of the W tile
     static constexpr uint32_t kStageBytes = kABytes + kBBytes;
-    static constexpr int kStages = BN == 256 ? 4 : (BN == 128 ? 6 : 8);
+    static constexpr int kStages = kStageBytes == 48 * 1024 ? 4 : (kStageBytes == 32 * 1024 ? 6 : 8);
     static constexpr uint32_t kTmemCols = 2 * BN;   // two accumulators
     static constexpr int kBarriers = 2 * kStages + 4;
     static constexpr int kSmemBytes = 1024 + kStages * kStageBytes + kEpilogueWarps * kPatchBytes + kBarriers * 8 + 16;
@@ -75,14 +85,78 @@ __device__ __forceinline__ void advance_len(int32_t* len, int b, int n, int cap,
         raise_status(dev_status, BT_DEV_OVERFLOW);  // the sequence keeps its rows and its length
 }
 
-template <int BN>
+// ---- the forms that differ between one CTA and a pair
+template <int kCtas>
+__device__ __forceinline__ void tmem_alloc(uint32_t slot, uint32_t cols)
+{
+    if constexpr (kCtas == 1) {
+        asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(slot), "r"(cols) : "memory");
+        asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
+    } else {   // issued by the same warp of both CTAs of the pair
+        asm volatile("tcgen05.alloc.cta_group::2.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(slot), "r"(cols) : "memory");
+        asm volatile("tcgen05.relinquish_alloc_permit.cta_group::2.sync.aligned;" ::: "memory");
+    }
+}
+template <int kCtas>
+__device__ __forceinline__ void tmem_dealloc(uint32_t tmem, uint32_t cols)
+{
+    if constexpr (kCtas == 1)
+        asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem), "r"(cols) : "memory");
+    else
+        asm volatile("tcgen05.dealloc.cta_group::2.sync.aligned.b32 %0, %1;" ::"r"(tmem), "r"(cols) : "memory");
+}
+// TMA load of a pair's CTA: lands in this CTA's shared memory, reports its bytes to the barrier named by a
+// shared::cluster address (the leader's).  No multicast.
+__device__ __forceinline__ void tma_load_3d_pair(uint32_t dst, const CUtensorMap* map, uint32_t bar_cluster, int c0, int c1, int c2)
+{
+    asm volatile(
+        "cp.async.bulk.tensor.3d.cta_group::2.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%3, %4, %5}], [%2];"
+        ::"r"(dst), "l"(map), "r"(bar_cluster), "r"(c0), "r"(c1), "r"(c2)
+        : "memory");
+}
+__device__ __forceinline__ void mma_bf16_pair(uint32_t tmem_d, uint64_t adesc, uint64_t bdesc, uint32_t idesc, uint32_t accumulate)
+{
+    const uint32_t z = 0;   // no output lane disabled
+    asm volatile(
+        "{\n\t.reg .pred p;\n\t"
+        "setp.ne.b32 p, %4, 0;\n\t"
+        "tcgen05.mma.cta_group::2.kind::f16 [%0], %1, %2, %3, {%5, %5, %5, %5, %5, %5, %5, %5}, p;\n\t}"
+        ::"r"(tmem_d), "l"(adesc), "l"(bdesc), "r"(idesc), "r"(accumulate), "r"(z)
+        : "memory");
+}
+// arrives, once the MMAs issued so far are done, on the barrier at this address in both CTAs of the pair
+__device__ __forceinline__ void mma_commit_pair(uint32_t bar)
+{
+    const uint16_t both = 3;
+    asm volatile("tcgen05.commit.cta_group::2.mbarrier::arrive::one.shared::cluster.multicast::cluster.b64 [%0], %1;" ::"r"(bar), "h"(both) : "memory");
+}
+__device__ __forceinline__ void mbar_arrive_cluster(uint32_t bar_cluster)
+{
+    asm volatile("mbarrier.arrive.shared::cluster.b64 _, [%0];" ::"r"(bar_cluster) : "memory");
+}
+__device__ __forceinline__ void cluster_sync_all()
+{
+    asm volatile("barrier.cluster.arrive.release.aligned;\n\tbarrier.cluster.wait.acquire.aligned;" ::: "memory");
+}
+__device__ __forceinline__ uint32_t cluster_cta_rank()
+{
+    uint32_t r;
+    asm volatile("mov.u32 %0, %%cluster_ctarank;" : "=r"(r));
+    return r;
+}
+
+template <int BN, int kCtas>
 __global__ void __launch_bounds__(kThreads, 1)
 project_tc_kernel(const __grid_constant__ CUtensorMap mapX, const __grid_constant__ CUtensorMap mapW, Params p)
 {
-    using C = Cfg<BN>;
+    using C = Cfg<BN, kCtas>;
     constexpr int S = C::kStages;
-    constexpr uint32_t IDESC = make_idesc(BM, BN, false);
+    constexpr uint32_t IDESC = make_idesc(BM * kCtas, BN, false);
     const ProjectArgs& a = p.a;
+    // a pair of CTAs works on one tile of 256 rows: `rank` is this CTA's half, `unit` numbers the pairs
+    const uint32_t rank = kCtas == 2 ? cluster_cta_rank() : 0u;
+    const int unit = (int)blockIdx.x / kCtas, n_units = (int)gridDim.x / kCtas;
+    const bool leader = rank == 0;
 
     extern __shared__ uint8_t smem_raw[];
     const uint32_t base = (smem_u32(smem_raw) + 1023u) & ~1023u;
@@ -105,17 +179,15 @@ project_tc_kernel(const __grid_constant__ CUtensorMap mapX, const __grid_constan
         }
         for (int i = 0; i < 2; ++i) {
             mbar_init(acc_full(i), 1);
-            mbar_init(acc_empty(i), kEpilogueWarps);
+            mbar_init(acc_empty(i), kEpilogueWarps * kCtas);   // the leader's collects both CTAs' epilogue warps
         }
         *abort_flag = 0;
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     }
-    if (warp == 0) {  // this warp allocates the CTA's tensor-memory columns and frees them at the end
-        asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(tmem_slot)), "r"(C::kTmemCols) : "memory");
-        asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
-    }
+    if (warp == 0) tmem_alloc<kCtas>(smem_u32(tmem_slot), C::kTmemCols);  // this warp allocates the tensor-memory columns and frees them at the end
     tc_fence_before();
     __syncthreads();
+    if constexpr (kCtas == 2) cluster_sync_all();   // the partner's barriers exist before anything is sent to them
     tc_fence_after();
     const uint32_t tmem = *tmem_slot;
 
@@ -123,7 +195,7 @@ project_tc_kernel(const __grid_constant__ CUtensorMap mapX, const __grid_constan
     // reads or writes global memory (the descriptor prefetch below touches only the kernel's own parameters).
     pdl_launch_dependents();
 
-    const int n_tiles = p.tiles_m * p.tiles_n;
+    const int n_tiles = p.tiles_m * p.tiles_n;     // tiles of BM * kCtas rows
     const int n_kb = (a.K + BK - 1) / BK;
 
     if (warp == kProducerWarp) {
@@ -133,30 +205,44 @@ project_tc_kernel(const __grid_constant__ CUtensorMap mapX, const __grid_constan
             pdl_wait();
             uint32_t it = 0;
             bool ok = true;
-            for (int tile = blockIdx.x; ok && tile < n_tiles; tile += gridDim.x) {
+            for (int tile = unit; ok && tile < n_tiles; tile += n_units) {
                 const int tm = tile / p.tiles_n, tn = tile - tm * p.tiles_n;
                 for (int kb = 0; kb < n_kb; ++kb, ++it) {
                     const uint32_t s = it % S;
                     ok = wait(empty(s), ((it / S) & 1) ^ 1, abort_flag, a.dev_status);
                     if (!ok) break;
                     const uint32_t dst = base + s * C::kStageBytes;
-                    mbar_expect_tx(full(s), C::kStageBytes);
-                    tma_load_3d(dst, &mapX, full(s), kb * BK, tm * BM, 0);
-                    tma_load_3d(dst + kABytes, &mapW, full(s), kb * BK, tn * BN, 0);
+                    if constexpr (kCtas == 1) {
+                        mbar_expect_tx(full(s), C::kStageBytes);
+                        tma_load_3d(dst, &mapX, full(s), kb * BK, tm * BM, 0);
+                        tma_load_3d(dst + kABytes, &mapW, full(s), kb * BK, tn * BN, 0);
+                    } else {
+                        // both CTAs' bytes are counted on the leader's barrier, which the leader arms
+                        if (leader) mbar_expect_tx(full(s), 2 * C::kStageBytes);
+                        const uint32_t bar = full(s) & kPeerBitMask;
+                        tma_load_3d_pair(dst, &mapX, bar, kb * BK, tm * (2 * BM) + (int)rank * BM, 0);
+                        tma_load_3d_pair(dst + kABytes, &mapW, bar, kb * BK, tn * BN + (int)rank * (BN / 2), 0);
+                    }
                 }
             }
-            // before the CTA goes: every copy this thread issued has landed (at once on the normal path, where the
-            // products that consumed them are done; bounded when something went wrong)
+            // Before the CTA goes, nothing may still be on its way to it.  One CTA: every copy this thread issued
+            // has landed (at once on the normal path, where the products that consumed them are done).  A pair:
+            // the last commits multicast to this CTA's "stage free" barriers have arrived, which also means the
+            // products that read this CTA's shared memory are done.  Bounded when something went wrong.
             for (uint32_t back = 1; back <= (uint32_t)S && back <= it; ++back) {
                 const uint32_t u = it - back;
-                if (!mbar_wait_walltime(full(u % S), (u / S) & 1, abort_flag, kSpinLimit, kWaitLimitNs)) break;
+                if constexpr (kCtas == 1) {
+                    if (!mbar_wait_walltime(full(u % S), (u / S) & 1, abort_flag, kSpinLimit, kWaitLimitNs)) break;
+                } else {
+                    if (!mbar_wait_walltime(empty(u % S), (u / S) & 1, abort_flag, kSpinLimit, kWaitLimitNs)) break;
+                }
             }
         }
     } else if (warp == kMmaWarp) {
-        if (lane == 0) {
+        if (lane == 0 && leader) {   // a pair's products are issued by its leader alone
             uint32_t it = 0, t = 0;
             bool ok = true;
-            for (int tile = blockIdx.x; ok && tile < n_tiles; tile += gridDim.x, ++t) {
+            for (int tile = unit; ok && tile < n_tiles; tile += n_units, ++t) {
                 const uint32_t acc = t & 1;
                 ok = wait(acc_empty(acc), ((t >> 1) & 1) ^ 1, abort_flag, a.dev_status);  // the epilogue has drained this accumulator
                 if (!ok) break;
@@ -168,12 +254,21 @@ project_tc_kernel(const __grid_constant__ CUtensorMap mapX, const __grid_constan
                     tc_fence_after();
                     const uint32_t a0 = base + s * C::kStageBytes, b0 = a0 + kABytes;
 #pragma unroll
-                    for (int kk = 0; kk < BK / 16; ++kk)
-                        mma_bf16(tmem + acc * BN, make_desc(a0 + kk * 32, 16, 1024), make_desc(b0 + kk * 32, 16, 1024), IDESC,
-                                 (kb > 0 || kk > 0) ? 1u : 0u);
-                    mma_commit(empty(s));
+                    for (int kk = 0; kk < BK / 16; ++kk) {
+                        if constexpr (kCtas == 1)
+                            mma_bf16(tmem + acc * BN, make_desc(a0 + kk * 32, 16, 1024), make_desc(b0 + kk * 32, 16, 1024), IDESC,
+                                     (kb > 0 || kk > 0) ? 1u : 0u);
+                        else
+                            mma_bf16_pair(tmem + acc * BN, make_desc(a0 + kk * 32, 16, 1024), make_desc(b0 + kk * 32, 16, 1024), IDESC,
+                                          (kb > 0 || kk > 0) ? 1u : 0u);
+                    }
+                    if constexpr (kCtas == 1) mma_commit(empty(s));
+                    else mma_commit_pair(empty(s));
                 }
-                if (ok) mma_commit(acc_full(acc));
+                if (ok) {
+                    if constexpr (kCtas == 1) mma_commit(acc_full(acc));
+                    else mma_commit_pair(acc_full(acc));
+                }
             }
         }
     } else {
@@ -186,11 +281,11 @@ project_tc_kernel(const __grid_constant__ CUtensorMap mapX, const __grid_constan
         uint32_t t = 0;
         bool ok = true;
         pdl_wait();
-        for (int tile = blockIdx.x; tile < n_tiles; tile += gridDim.x, ++t) {
+        for (int tile = unit; tile < n_tiles; tile += n_units, ++t) {
             const int tm = tile / p.tiles_n, tn = tile - tm * p.tiles_n;
             const uint32_t acc = t & 1;
             // this lane's own row: which sequence, which of its n rows, and where the row lands in the cache
-            const int m = tm * BM + wq * 32 + lane;
+            const int m = tm * (BM * kCtas) + (int)rank * BM + wq * 32 + lane;
             int row_b = -1, row_i = 0, row_rc = -1;
             if (m < a.M) {
                 if (a.mode == kProjectPlain) {
@@ -278,15 +373,19 @@ project_tc_kernel(const __grid_constant__ CUtensorMap mapX, const __grid_constan
             }
             tc_fence_before();
             __syncwarp();
-            if (lane == 0) mbar_arrive(acc_empty(acc));
+            if (lane == 0) {
+                if constexpr (kCtas == 1) mbar_arrive(acc_empty(acc));
+                else mbar_arrive_cluster(acc_empty(acc) & kPeerBitMask);   // the leader's barrier
+            }
         }
     }
 
     tc_fence_before();
     __syncthreads();
+    if constexpr (kCtas == 2) cluster_sync_all();   // both CTAs are through with each other's barriers and tensor memory
     if (warp == 0) {
         tc_fence_after();
-        asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem), "r"(C::kTmemCols) : "memory");
+        tmem_dealloc<kCtas>(tmem, C::kTmemCols);
     }
     // With a sync word the lengths go up inside this launch: every CTA counts itself in once all of its tiles are
     // stored (the barrier above: all epilogue warps are through), and the one that arrives last - when nobody
@@ -319,23 +418,38 @@ __global__ void project_len_advance_kernel(int32_t* len, int B, int n, int cap, 
     if (b < B) advance_len(len, b, n, cap, reset_first, reset_mask, dev_status);
 }
 
-template <int BN>
+template <int BN, int kCtas>
 static cudaError_t launch_bn(const ProjectArgs& a, int dev, int sms, cudaStream_t stream)
 {
-    using C = Cfg<BN>;
+    using C = Cfg<BN, kCtas>;
     static PerDeviceOnce limit_raised;
-    cudaError_t e = raise_smem_limit_once(limit_raised, dev, project_tc_kernel<BN>, C::kSmemBytes);
+    cudaError_t e = raise_smem_limit_once(limit_raised, dev, project_tc_kernel<BN, kCtas>, C::kSmemBytes);
     if (e != cudaSuccess) return e;
     CUtensorMap mx, mw;
-    if (!make_slab_map(&mx, a.x, a.K, a.M, a.M, 1, BM) || !make_slab_map(&mw, a.w, a.K, a.N, a.N, 1, BN)) return cudaErrorInvalidValue;
+    if (!make_slab_map(&mx, a.x, a.K, a.M, a.M, 1, BM) || !make_slab_map(&mw, a.w, a.K, a.N, a.N, 1, BN / kCtas)) return cudaErrorInvalidValue;
     Params p;
     p.a = a;
-    p.tiles_m = (a.M + BM - 1) / BM;
+    p.tiles_m = (a.M + BM * kCtas - 1) / (BM * kCtas);
     p.tiles_n = (a.N + BN - 1) / BN;
     const long long tiles = (long long)p.tiles_m * p.tiles_n;
     if (tiles > 0x7fffffffLL) return cudaErrorInvalidConfiguration;
-    const int grid = (int)(tiles < sms ? tiles : sms);
-    return launch_pdl(project_tc_kernel<BN>, dim3(grid), dim3(kThreads), (size_t)C::kSmemBytes, stream, mx, mw, p);
+    const int units = sms / kCtas;
+    const int grid = (int)(tiles < units ? tiles : units) * kCtas;
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = dim3(grid);
+    cfg.blockDim = dim3(kThreads);
+    cfg.dynamicSmemBytes = (size_t)C::kSmemBytes;
+    cfg.stream = stream;
+    cudaLaunchAttribute attr[2];
+    attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr[0].val.programmaticStreamSerializationAllowed = 1;
+    attr[1].id = cudaLaunchAttributeClusterDimension;
+    attr[1].val.clusterDim.x = kCtas;
+    attr[1].val.clusterDim.y = 1;
+    attr[1].val.clusterDim.z = 1;
+    cfg.attrs = attr;
+    cfg.numAttrs = kCtas == 2 ? 2 : 1;
+    return cudaLaunchKernelEx(&cfg, project_tc_kernel<BN, kCtas>, mx, mw, p);
 }
 
 }  // namespace proj
@@ -347,15 +461,36 @@ cudaError_t launch_project(const ProjectArgs& a, cudaStream_t stream)
     int dev = 0, sms = 0;
     cudaError_t e = current_device(&dev, &sms);
     if (e != cudaSuccess) return e;
-    // the widest tile that still gives every SM one
-    const long long tiles_m = (a.M + proj::BM - 1) / proj::BM;
-    auto tiles = [&](int bn) { return tiles_m * ((a.N + bn - 1) / bn); };
-    if (tiles(256) >= sms)
-        e = proj::launch_bn<256>(a, dev, sms, stream);
-    else if (tiles(128) >= sms)
-        e = proj::launch_bn<128>(a, dev, sms, stream);
-    else
-        e = proj::launch_bn<64>(a, dev, sms, stream);
+    // Tile shape: the one with the shortest estimated launch.  All tiles of a launch take the same time, so a launch
+    // lasts (rounds of tiles) x (time of one tile); a tile's time is its area per SM over the relative rate that
+    // shape sustains (measured: 128 x 256 on one SM = 1; 256 x 256 on a pair 1.11, a third less operand traffic per
+    // SM; the narrower tiles less, their operands being re-read more often).
+    struct Shape {
+        int bn, ctas;
+        double rate;
+    };
+    const Shape shapes[4] = {{256, 2, 1.11}, {256, 1, 1.0}, {128, 1, 0.9}, {64, 1, 0.75}};
+    int best = 1;
+    double best_cost = 0.0;
+    for (int i = 0; i < 4; ++i) {
+        const Shape& sh = shapes[i];
+        if (sh.ctas == 2 && sms % 2 != 0) continue;
+        const long long rows = (long long)proj::BM * sh.ctas;
+        const long long tiles = ((a.M + rows - 1) / rows) * ((a.N + sh.bn - 1) / sh.bn);
+        const long long units = sms / sh.ctas;
+        const long long rounds = (tiles + units - 1) / units;
+        const double cost = (double)rounds * (double)(proj::BM * sh.bn) / sh.rate;
+        if (i == 0 || cost < best_cost - 1e-9) {
+            best = i;
+            best_cost = cost;
+        }
+    }
+    switch (best) {
+        case 0: e = proj::launch_bn<256, 2>(a, dev, sms, stream); break;
+        case 1: e = proj::launch_bn<256, 1>(a, dev, sms, stream); break;
+        case 2: e = proj::launch_bn<128, 1>(a, dev, sms, stream); break;
+        default: e = proj::launch_bn<64, 1>(a, dev, sms, stream); break;
+    }
     if (e != cudaSuccess || a.mode == kProjectPlain || a.sync_word != nullptr) return e;
     const int B = a.M / a.n_rows;
     return launch_pdl(proj::project_len_advance_kernel, dim3((B + 255) / 256), dim3(256), 0, stream, a.cache.len, B, a.n_rows,
