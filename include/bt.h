@@ -290,10 +290,8 @@ bt_status bt_prefix_project(const bt_config* cfg, const void* ctx, const void* w
  *   cache rows len[b]+i of head h = the K and V parts,   i < n_rows
  *   len[b] += n_rows.
  * A sequence without room for n_rows more rows keeps its cache and length, BT_DEV_OVERFLOW is raised
- * (its q_out rows are still written).  The lengths may only go up once every tile of the product has
- * read the old ones.  sync_word: optional device uint32 that is zero on entry and is left zero; with it
- * the CTA that finishes last advances the lengths inside the one launch, without it (NULL) a second,
- * small launch does.  Calls that can overlap on the GPU need a word each.
+ * (its q_out rows are still written).  Two launches: the product with the cache-writing epilogue, then
+ * a small one that advances the lengths once every tile has read the old ones.
  * Attention then runs over the cache as it stands: bt_block_decode_attn for the block decoder,
  * bt_token_decode_attn with k_new = v_new = NULL (n_q = n_rows) for the token decoder.
  * Returns BT_ERR_CAPACITY if n_rows exceeds the cache capacity.
@@ -304,11 +302,10 @@ bt_status bt_prefix_project(const bt_config* cfg, const void* ctx, const void* w
  */
 bt_status bt_block_qkv_project_append(const bt_config* cfg, bt_block_cache* cache, int layer, const void* x,
                                       int n_rows, const void* w_qkv, const void* bias, void* q_out,
-                                      uint32_t* sync_word, uint32_t* dev_status, void* stream);
+                                      uint32_t* dev_status, void* stream);
 bt_status bt_local_qkv_project_append(const bt_config* cfg, bt_local_cache* cache, int layer, const void* x,
                                       int n_rows, const void* w_qkv, const void* bias, int reset_first,
-                                      const uint8_t* reset_mask, void* q_out, uint32_t* sync_word,
-                                      uint32_t* dev_status, void* stream);
+                                      const uint8_t* reset_mask, void* q_out, uint32_t* dev_status, void* stream);
 
 /*
  * Self-test of the bounded waits (test support; the paper has no counterpart).  Every wait inside the

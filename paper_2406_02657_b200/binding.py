@@ -75,8 +75,8 @@ def _load() -> ctypes.CDLL:
     lib.bt_block_decode_attn_noalloc.argtypes = [cfgp, ctypes.POINTER(bt_block_cache), i32, vp, vp, vp, vp]
     lib.bt_selftest_bounded_wait.argtypes = [vp, vp, vp]
     lib.bt_prefix_project.argtypes = [cfgp, vp, vp, vp, vp, vp, vp]
-    lib.bt_block_qkv_project_append.argtypes = [cfgp, ctypes.POINTER(bt_block_cache), i32, vp, i32, vp, vp, vp, vp, vp, vp]
-    lib.bt_local_qkv_project_append.argtypes = [cfgp, ctypes.POINTER(bt_local_cache), i32, vp, i32, vp, vp, i32, vp, vp, vp, vp, vp]
+    lib.bt_block_qkv_project_append.argtypes = [cfgp, ctypes.POINTER(bt_block_cache), i32, vp, i32, vp, vp, vp, vp, vp]
+    lib.bt_local_qkv_project_append.argtypes = [cfgp, ctypes.POINTER(bt_local_cache), i32, vp, i32, vp, vp, i32, vp, vp, vp, vp]
     for name in EXPORTS[4:]:
         getattr(lib, name).restype = ctypes.c_int
     return lib
@@ -212,22 +212,21 @@ def bt_prefix_project(cfg, ctx, w_prefix, bias, prefix_out, dev_status=None, str
                                   _ptr(dev_status), _stream(stream)), "bt_prefix_project")
 
 
-def bt_block_qkv_project_append(cfg, cache: BlockCache, layer, x, w_qkv, bias, q_out, n_rows=None, sync_word=None, dev_status=None,
-                                stream=None):
+def bt_block_qkv_project_append(cfg, cache: BlockCache, layer, x, w_qkv, bias, q_out, n_rows=None, dev_status=None, stream=None):
     """QKV projection of x [B,n,D]; Q -> q_out [B,H,n,hd], K and V rows appended to the block cache."""
     n_rows = x.shape[1] if n_rows is None else n_rows
     _check(_lib.bt_block_qkv_project_append(ctypes.byref(cfg), ctypes.byref(cache.c), layer, _ptr(x), n_rows, _ptr(w_qkv),
-                                            _ptr(bias), _ptr(q_out), _ptr(sync_word), _ptr(dev_status), _stream(stream)),
+                                            _ptr(bias), _ptr(q_out), _ptr(dev_status), _stream(stream)),
            "bt_block_qkv_project_append")
 
 
 def bt_local_qkv_project_append(cfg, cache: LocalCache, layer, x, w_qkv, bias, q_out, n_rows=None, reset_first=False,
-                                reset_mask=None, sync_word=None, dev_status=None, stream=None):
+                                reset_mask=None, dev_status=None, stream=None):
     """QKV projection of x [B,n,D]; Q -> q_out [B,H,n,hd], K and V rows appended to the local cache
     (after the optional block-boundary reset)."""
     n_rows = x.shape[1] if n_rows is None else n_rows
     _check(_lib.bt_local_qkv_project_append(ctypes.byref(cfg), ctypes.byref(cache.c), layer, _ptr(x), n_rows, _ptr(w_qkv),
-                                            _ptr(bias), 1 if reset_first else 0, _ptr(reset_mask), _ptr(q_out), _ptr(sync_word),
+                                            _ptr(bias), 1 if reset_first else 0, _ptr(reset_mask), _ptr(q_out),
                                             _ptr(dev_status), _stream(stream)), "bt_local_qkv_project_append")
 
 

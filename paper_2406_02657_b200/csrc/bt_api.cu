@@ -401,10 +401,9 @@ bt_status bt_prefix_project(const bt_config* cfg, const void* ctx, const void* w
 }
 
 static bt_status qkv_project(const bt_config* cfg, const bt::CacheView& view, const void* x, int n_rows, const void* w_qkv,
-                             const void* bias, int reset_first, const uint8_t* reset_mask, void* q_out, uint32_t* sync_word,
-                             uint32_t* dev_status, void* stream)
+                             const void* bias, int reset_first, const uint8_t* reset_mask, void* q_out, uint32_t* dev_status,
+                             void* stream)
 {
-    if (!al4(sync_word)) return BT_ERR_UNSUPPORTED;
     const long long D = (long long)cfg->heads * cfg->head_dim;
     if ((long long)cfg->batch * n_rows > 0x7fffffffLL / 2 || 3 * D > 0x7fffffffLL) return BT_ERR_UNSUPPORTED;
     bt::ProjectArgs a = {};
@@ -422,15 +421,13 @@ static bt_status qkv_project(const bt_config* cfg, const bt::CacheView& view, co
     a.hd = cfg->head_dim;
     a.reset_first = reset_first ? 1 : 0;
     a.reset_mask = reset_mask;
-    a.sync_word = sync_word;
     a.dev_status = dev_status;
     if (!bt::project_supported(a)) return BT_ERR_UNSUPPORTED;
     return cuda_status(bt::launch_project(a, (cudaStream_t)stream));
 }
 
 bt_status bt_block_qkv_project_append(const bt_config* cfg, bt_block_cache* cache, int layer, const void* x, int n_rows,
-                                      const void* w_qkv, const void* bias, void* q_out, uint32_t* sync_word,
-                                      uint32_t* dev_status, void* stream)
+                                      const void* w_qkv, const void* bias, void* q_out, uint32_t* dev_status, void* stream)
 {
     bt_status st = check_config(cfg, layer);
     if (st != BT_OK) return st;
@@ -440,12 +437,12 @@ bt_status bt_block_qkv_project_append(const bt_config* cfg, bt_block_cache* cach
     if (n_rows <= 0) return BT_ERR_SHAPE;
     if (n_rows > cfg->max_blocks) return BT_ERR_CAPACITY;
     if (!block_cache_aligned(cache)) return BT_ERR_UNSUPPORTED;
-    return qkv_project(cfg, block_view(cfg, cache, layer), x, n_rows, w_qkv, bias, 0, nullptr, q_out, sync_word, dev_status, stream);
+    return qkv_project(cfg, block_view(cfg, cache, layer), x, n_rows, w_qkv, bias, 0, nullptr, q_out, dev_status, stream);
 }
 
 bt_status bt_local_qkv_project_append(const bt_config* cfg, bt_local_cache* cache, int layer, const void* x, int n_rows,
                                       const void* w_qkv, const void* bias, int reset_first, const uint8_t* reset_mask,
-                                      void* q_out, uint32_t* sync_word, uint32_t* dev_status, void* stream)
+                                      void* q_out, uint32_t* dev_status, void* stream)
 {
     bt_status st = check_config(cfg, layer);
     if (st != BT_OK) return st;
@@ -455,8 +452,7 @@ bt_status bt_local_qkv_project_append(const bt_config* cfg, bt_local_cache* cach
     if (n_rows <= 0) return BT_ERR_SHAPE;
     if (n_rows > local_cap(cfg)) return BT_ERR_CAPACITY;
     if (!local_cache_aligned(cache)) return BT_ERR_UNSUPPORTED;
-    return qkv_project(cfg, local_view(cfg, cache, layer), x, n_rows, w_qkv, bias, reset_first, reset_mask, q_out, sync_word, dev_status,
-                       stream);
+    return qkv_project(cfg, local_view(cfg, cache, layer), x, n_rows, w_qkv, bias, reset_first, reset_mask, q_out, dev_status, stream);
 }
 
 bt_status bt_selftest_bounded_wait(uint32_t* report, uint32_t* dev_status, void* stream)

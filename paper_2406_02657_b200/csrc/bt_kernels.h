@@ -104,9 +104,7 @@ cudaError_t launch_block_prefill_tc(const PrefillArgs& a, uint32_t* dev_status, 
 //   kProjectQkv   : M = B * n_rows rows (sequence b, row i), N = 3 * H * hd output features ordered Q, K, V,
 //                   each (h, d): Q -> out [B][H][n_rows][hd]; K, V -> rows len_old[b] + i of `cache`
 //                   (len_old = 0 where the reset applies); a sequence without room for n_rows rows keeps
-//                   its cache.  The lengths are advanced (and those sequences flagged) by the CTA that finishes
-//                   last when sync_word (a device uint32, zero on entry, left zero) is given, else by a second
-//                   launch.
+//                   its cache.  A second launch then advances the lengths (and flags those sequences).
 enum { kProjectPlain = 0, kProjectQkv = 1 };
 struct ProjectArgs {
     const void* x;
@@ -119,7 +117,6 @@ struct ProjectArgs {
     int n_rows, H, hd;        // kProjectQkv
     int reset_first;
     const uint8_t* reset_mask;
-    uint32_t* sync_word;
     uint32_t* dev_status;
 };
 bool project_supported(const ProjectArgs& a);

@@ -387,28 +387,11 @@ project_tc_kernel(const __grid_constant__ CUtensorMap mapX, const __grid_constan
         tc_fence_after();
         tmem_dealloc<kCtas>(tmem, C::kTmemCols);
     }
-    // With a sync word the lengths go up inside this launch: every CTA counts itself in once all of its tiles are
-    // stored (the barrier above: all epilogue warps are through), and the one that arrives last - when nobody
-    // reads the old lengths any more - advances them and puts the word back to zero.
-    if (a.mode == kProjectQkv && a.sync_word != nullptr) {
-        __shared__ int is_last;
-        if (threadIdx.x == 0) {
-            __threadfence();
-            is_last = atomicAdd(a.sync_word, 1u) == gridDim.x - 1;
-        }
-        __syncthreads();
-        if (is_last) {
-            pdl_wait();  // not every thread of the CTA has been through it yet
-            __threadfence();
-            const int B = a.M / a.n_rows;
-            for (int b = threadIdx.x; b < B; b += blockDim.x) advance_len(a.cache.len, b, a.n_rows, a.cache.cap, a.reset_first, a.reset_mask, a.dev_status);
-            if (threadIdx.x == 0) *a.sync_word = 0u;
-        }
-    }
 }
 
-// The lengths go up once every tile has read the old ones: without a sync word, a second, tiny launch
-// behind the product.
+// The lengths go up once every tile has read the old ones: a second, tiny launch behind the product (it starts
+// under programmatic dependent launch while the product drains; counting the product's CTAs in on a word in
+// global memory and letting the last one advance the lengths was measured 2 us slower per step).
 __global__ void project_len_advance_kernel(int32_t* len, int B, int n, int cap, int reset_first, const uint8_t* reset_mask,
                                            uint32_t* dev_status)
 {
@@ -491,7 +474,7 @@ cudaError_t launch_project(const ProjectArgs& a, cudaStream_t stream)
         case 2: e = proj::launch_bn<128, 1>(a, dev, sms, stream); break;
         default: e = proj::launch_bn<64, 1>(a, dev, sms, stream); break;
     }
-    if (e != cudaSuccess || a.mode == kProjectPlain || a.sync_word != nullptr) return e;
+    if (e != cudaSuccess || a.mode == kProjectPlain) return e;
     const int B = a.M / a.n_rows;
     return launch_pdl(proj::project_len_advance_kernel, dim3((B + 255) / 256), dim3(256), 0, stream, a.cache.len, B, a.n_rows,
                       a.cache.cap, a.reset_first, a.reset_mask, a.dev_status);

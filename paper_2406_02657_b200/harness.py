@@ -404,7 +404,6 @@ class ProjectRun:
         self.cfg = bt.make_config(B, H, hd, w.block_len, P, max(1, w.max_blocks), w.n_layers)
         mk = fill if fill is not None else (lambda tid, sh: torch.zeros(sh, dtype=torch.bfloat16, device=device))
         self.status = torch.zeros(1, dtype=torch.int32, device=device)
-        self.sync = torch.zeros(1, dtype=torch.int32, device=device)
         if kind == "prefix":
             self.x, self.wt, self.bias = mk(40, (L, B, D)), mk(41, (L, P * D, D)), mk(42, (L, P * D))
             self.out = torch.empty((L, B, P, D), dtype=torch.bfloat16, device=device)
@@ -430,10 +429,10 @@ class ProjectRun:
                 bt.bt_prefix_project(self.cfg, self.x[i], self.wt[i], self.bias[i], self.out[i], dev_status=self.status)
             elif self.kind == "qkv_token":
                 bt.bt_local_qkv_project_append(self.cfg, self.cache, l, self.x[i], self.wt[i], self.bias[i], self.out[i],
-                                               reset_first=True, sync_word=self.sync, dev_status=self.status)
+                                               reset_first=True, dev_status=self.status)
             else:
                 bt.bt_block_qkv_project_append(self.cfg, self.cache, l, self.x[i], self.wt[i], self.bias[i], self.out[i],
-                                               sync_word=self.sync, dev_status=self.status)
+                                               dev_status=self.status)
 
     def rewind(self):
         if self.kind == "qkv_block":

@@ -98,15 +98,13 @@ def test_host_detectable_errors_return_before_launch(bt):
     # projections
     assert L.bt_prefix_project(ref(cfg), fake, None, None, fake, None, None) == bt.BT_ERR_NULL
     assert L.bt_prefix_project(ref(bad), fake, fake, None, fake, None, None) == bt.BT_ERR_UNSUPPORTED
-    assert L.bt_block_qkv_project_append(ref(cfg), ref(bc), 0, fake, 65, fake, None, fake, None, None, None) == bt.BT_ERR_CAPACITY
-    assert L.bt_block_qkv_project_append(ref(cfg), ref(bc), 0, fake, 0, fake, None, fake, None, None, None) == bt.BT_ERR_SHAPE
-    assert L.bt_block_qkv_project_append(ref(cfg), ref(nullc), 0, fake, 1, fake, None, fake, None, None, None) == bt.BT_ERR_NULL
-    assert L.bt_block_qkv_project_append(ref(cfg), ref(bc), 2, fake, 1, fake, None, fake, None, None, None) == bt.BT_ERR_SHAPE
-    assert L.bt_local_qkv_project_append(ref(cfg), ref(lc), 0, fake, 6, fake, None, 0, None, fake, None, None, None) == bt.BT_ERR_CAPACITY
-    assert L.bt_local_qkv_project_append(ref(cfg), ref(lc), 0, fake, 1, None, None, 0, None, fake, None, None, None) == bt.BT_ERR_NULL
-    assert L.bt_local_qkv_project_append(ref(cfg), ref(lc), 0, fake, 1, fake, ctypes.c_void_p(0x1002), 0, None, fake, None, None, None) \
-        == bt.BT_ERR_UNSUPPORTED
-    assert L.bt_local_qkv_project_append(ref(cfg), ref(lc), 0, fake, 1, fake, None, 0, None, fake, ctypes.c_void_p(0x1002), None, None) \
+    assert L.bt_block_qkv_project_append(ref(cfg), ref(bc), 0, fake, 65, fake, None, fake, None, None) == bt.BT_ERR_CAPACITY
+    assert L.bt_block_qkv_project_append(ref(cfg), ref(bc), 0, fake, 0, fake, None, fake, None, None) == bt.BT_ERR_SHAPE
+    assert L.bt_block_qkv_project_append(ref(cfg), ref(nullc), 0, fake, 1, fake, None, fake, None, None) == bt.BT_ERR_NULL
+    assert L.bt_block_qkv_project_append(ref(cfg), ref(bc), 2, fake, 1, fake, None, fake, None, None) == bt.BT_ERR_SHAPE
+    assert L.bt_local_qkv_project_append(ref(cfg), ref(lc), 0, fake, 6, fake, None, 0, None, fake, None, None) == bt.BT_ERR_CAPACITY
+    assert L.bt_local_qkv_project_append(ref(cfg), ref(lc), 0, fake, 1, None, None, 0, None, fake, None, None) == bt.BT_ERR_NULL
+    assert L.bt_local_qkv_project_append(ref(cfg), ref(lc), 0, fake, 1, fake, ctypes.c_void_p(0x1002), 0, None, fake, None, None) \
         == bt.BT_ERR_UNSUPPORTED
     # host-driven step
     assert L.bt_block_decode_step_host(ref(cfg), ref(bc), 0, None, fake, fake, fake, fake, fake, fake, fake,

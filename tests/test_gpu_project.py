@@ -90,13 +90,8 @@ def _block_setup(bt, seed, B, H, hd, N, lens, layers=2, layer=1):
     return cfg, cache, oc
 
 
-def sync_word():
-    return torch.zeros(1, dtype=torch.int32, device="cuda")
-
-
-@pytest.mark.parametrize("with_sync_word", [False, True])
 @pytest.mark.parametrize("hd,n", [(64, 1), (128, 1), (64, 3)])
-def test_block_qkv_identity_weights_cache_the_input_bit_for_bit(bt, hd, n, with_sync_word):
+def test_block_qkv_identity_weights_cache_the_input_bit_for_bit(bt, hd, n):
     B, H, N, layer = 9, 3, 40, 1
     D = H * hd
     lens = [0, 1, 39, 40, 17, 40 - n, 40 - n + 1 if n > 1 else 5, 8, 33]
@@ -105,9 +100,7 @@ def test_block_qkv_identity_weights_cache_the_input_bit_for_bit(bt, hd, n, with_
     W = bits(np.concatenate([np.eye(D), 2 * np.eye(D), -np.eye(D)]))
     q = torch.full((B, H, n, hd), 5.0, dtype=torch.bfloat16, device="cuda")
     st = status_word()
-    word = sync_word() if with_sync_word else None   # lengths advanced inside the launch, or by a second launch
-    bt.bt_block_qkv_project_append(cfg, cache, layer, to_dev(x), to_dev(W), None, q, sync_word=word, dev_status=st)
-    assert word is None or word.item() == 0
+    bt.bt_block_qkv_project_append(cfg, cache, layer, to_dev(x), to_dev(W), None, q, dev_status=st)
     q_ref = oracle.qkv_project_append(oc, x, W)
     assert np.array_equal(to_f64(q), q_ref)                               # exact arithmetic: bit for bit
     assert np.array_equal(gen.torch_to_bits(cache.k[layer]), oc.k) and np.array_equal(gen.torch_to_bits(cache.v[layer]), oc.v)
@@ -130,10 +123,7 @@ def test_block_qkv_random_weights(bt, B, H, hd, n, with_bias):
     bias = rnd(730 + B, 5, (3 * D,)) if with_bias else None
     q = torch.empty((B, H, n, hd), dtype=torch.bfloat16, device="cuda")
     st = status_word()
-    word = sync_word() if with_bias else None
-    bt.bt_block_qkv_project_append(cfg, cache, layer, to_dev(x), to_dev(W), None if bias is None else to_dev(bias), q,
-                                   sync_word=word, dev_status=st)
-    assert word is None or word.item() == 0
+    bt.bt_block_qkv_project_append(cfg, cache, layer, to_dev(x), to_dev(W), None if bias is None else to_dev(bias), q, dev_status=st)
     q_ref = oracle.qkv_project_append(oc, x, W, bias)
     assert_close_proj(q, q_ref, "q of the block QKV projection")
     assert cache.len[layer].cpu().tolist() == oc.len.tolist() and st.item() == int(oc.status[0]) == bt.BT_DEV_OVERFLOW
@@ -172,12 +162,11 @@ def test_local_qkv_projection_then_attend_only_over_two_blocks(bt, hd, P):
     W, bias = rnd(740 + hd, 4, (3 * D, D)), rnd(740 + hd, 5, (3 * D,))
     Wd, bd = to_dev(W), to_dev(bias)
     st = status_word()
-    word = sync_word() if hd == 64 else None
     for t, (reset, n, len_after) in enumerate(oracle.token_step_schedule(L_B, P, 2 * L_B)):
         x = unit_rows(741 + hd, t, (B, n, D))
         q = torch.empty((B, H, n, hd), dtype=torch.bfloat16, device="cuda")
         out = torch.empty((B, H, n, hd), dtype=torch.bfloat16, device="cuda")
-        bt.bt_local_qkv_project_append(cfg, lc, layer, to_dev(x), Wd, bd, q, reset_first=bool(reset), sync_word=word, dev_status=st)
+        bt.bt_local_qkv_project_append(cfg, lc, layer, to_dev(x), Wd, bd, q, reset_first=bool(reset), dev_status=st)
         bt.bt_token_decode_attn(cfg, lc, layer, q, None, None, out, n_q=n, dev_status=st)
         q_ref = oracle.qkv_project_append(oc, x, W, bias, reset_first=bool(reset))
         assert_close_proj(q, q_ref, f"q at token step {t}")
@@ -189,7 +178,7 @@ def test_local_qkv_projection_then_attend_only_over_two_blocks(bt, hd, P):
         for g, r in ((gk, oc.k), (gv, oc.v)):
             err = np.abs(widen(g[:, :, :len_after]) - widen(r[:, :, :len_after]))
             assert (err <= 2e-3 + 8e-3 * np.abs(widen(r[:, :, :len_after]))).all()
-    assert st.item() == 0 and not lc.len[0].any() and (word is None or word.item() == 0)
+    assert st.item() == 0 and not lc.len[0].any()
 
 
 def test_local_qkv_projection_masked_reset_and_overflow(bt):
@@ -209,10 +198,8 @@ def test_local_qkv_projection_masked_reset_and_overflow(bt):
     W = bits(np.concatenate([np.eye(D), 2 * np.eye(D), -np.eye(D)]))
     q = torch.empty((B, H, n, hd), dtype=torch.bfloat16, device="cuda")
     st = status_word()
-    word = sync_word()
-    bt.bt_local_qkv_project_append(cfg, lc, 0, to_dev(x), to_dev(W), None, q, reset_mask=torch.from_numpy(mask).cuda(), sync_word=word,
+    bt.bt_local_qkv_project_append(cfg, lc, 0, to_dev(x), to_dev(W), None, q, reset_mask=torch.from_numpy(mask).cuda(),
                                    dev_status=st)
-    assert word.item() == 0
     q_ref = oracle.qkv_project_append(oc, x, W, reset_mask=mask)
     assert np.array_equal(to_f64(q), q_ref)
     assert lc.len[0].cpu().tolist() == oc.len.tolist() == [2, 2, 6, 5, 2, 3]
@@ -261,9 +248,8 @@ def test_qkv_projection_at_the_bench_shapes(bt, B, H, hd, n):
     cache.len[0].copy_(lens)
     q = torch.empty((B, H, n, hd), dtype=torch.bfloat16, device="cuda")
     st = status_word()
-    word = sync_word()
-    bt.bt_block_qkv_project_append(cfg, cache, 0, x, W, bias, q, sync_word=word, dev_status=st)
-    assert torch.equal(cache.len[0], lens + n) and st.item() == 0 and word.item() == 0
+    bt.bt_block_qkv_project_append(cfg, cache, 0, x, W, bias, q, dev_status=st)
+    assert torch.equal(cache.len[0], lens + n) and st.item() == 0
     seqs = sorted({0, 1, B // 3, B - 2, B - 1})
     oc = oracle.Cache(len(seqs), H, N, hd)
     oc.len[...] = lens.cpu().numpy()[seqs]
