@@ -219,6 +219,11 @@ def workload_config(w, name):
         c.update(workload="qkv_project_block: QKV projection of one block step at the shape of configs[1] (256 rows, model dim 1024), "
                           "K and V rows appended to the block cache by the epilogue, distinct weights per layer",
                  l2="no flush: the steps rotate over independent sets of inputs, weights and outputs, 288 MB per graph replay")
+    elif name == "token_decode_projected":
+        c.update(workload="token_decode_projected: configs[2] with the QKV projection in the path - per layer and token step, x [4096,1,1024] is "
+                          "projected, K and V rows go into the local cache from the product's epilogue, the attention call attends over the "
+                          "cache as it stands; 3 launches per layer and step (product, length update, attention)",
+                 l2="no flush: inputs rotate over a ring larger than L2")
     elif name == "prefix_project":
         c.update(workload="prefix_project: context embedding -> P prefix embeddings for 4096 sequences, model dim 1024, 12 distinct weight sets",
                  l2="no flush: 250 MB per step")
@@ -397,6 +402,26 @@ def measure(name, w, args, env, primary):
                 for (reset, _, _), (q, k, v) in zip(sched, ins):
                     oracle.token_decode_attn(oc, q, k, v, reset_first=bool(reset))
             cpu = oracle_sample(go, n_seq * n_st / w.n_layers, f"{n_seq} of {w.batch} sequences x 1 of {w.n_layers} layers x {n_st} token steps")
+    elif name == "token_decode_projected":
+        run = harness.ProjectedTokenRun(w, fill=fill)
+        n_tok = run.capture()
+        tokens_per_step = w.batch * n_tok
+        sampler.start()
+        ms = timer(run.replay, steps, warmup)
+        clocks = sampler.stop()
+        assert run.status.item() == 0
+        D = w.heads * w.head_dim
+        # per layer and step: the product's bytes (x, W, bias in; q, K row, V row out) + the attention's (q in, the
+        # j + 1 cached rows in, out out); the new K,V rows are written once, by the product
+        row = w.head_dim * traffic.BF16
+        attn = sum(w.batch * w.heads * (2 * row + (P + j) * 2 * row) for j in range(w.block_len)) / w.block_len
+        alg = traffic.linear_bytes(w.batch, 3 * D, D) + attn
+        fl = traffic.linear_flops(w.batch, 3 * D, D)
+        n_layer_steps = w.n_layers * n_tok
+        roof = hbm_roofline(pk, "project_tc_kernel + token_step_pipelined_kernel (one layer of one token step)", alg,
+                            ms / n_layer_steps, n_layer_steps * alg, ms, None)
+        add_tensor_roofline(roof, pk, fl, alg, ms / n_layer_steps, in_long_step=False)
+        launches = run.launches_per_step * n_tok * steps
     elif name == "sweep":
         # a step = one whole generation: prompt prefill + bulk append, then gen_tokens / L_B generated blocks
         # (CUDA-graph replays of `ring` blocks each); tokens = batch x generated tokens
@@ -491,6 +516,7 @@ SECONDARY = [
     # step counts sized for about half a second of timed work each, so that the clock sampler sees the region
     ("token_decode", 1, 0, 400, 3), ("token_decode", 2, 0, 300, 3), ("token_decode", 8, 0, 150, 3), ("block_prefill", 0, 0, 600, 3), ("block_prefill_8k", 0, 0, 250, 3),
     ("qkv_project_token", 0, 0, 1200, 3), ("qkv_project_block", 0, 0, 2000, 3), ("prefix_project", 0, 0, 2000, 3),
+    ("token_decode_projected", 0, 0, 120, 3),
     ("sweep", 0, 4, 2, 1), ("sweep", 0, 8, 2, 1),
 ]
 
@@ -557,7 +583,7 @@ def main():
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--workload", default="block_decode",
                     choices=["block_decode", "block_decode_16k", "dense_decode", "token_decode", "block_prefill", "block_prefill_8k", "sweep",
-                             "qkv_project_token", "qkv_project_block", "prefix_project"])
+                             "qkv_project_token", "qkv_project_block", "prefix_project", "token_decode_projected"])
     ap.add_argument("--no-secondary", action="store_true", help="default workload only: skip the shorter runs of the other configurations")
     ap.add_argument("--block-len", type=int, default=4, help="L_B of the generation sweep (1, 2, 4 or 8)")
     ap.add_argument("--prefix-len", type=int, default=0, help="prefix length P (token_decode: default 1 = benchmark configs[2], 2 = the paper's main setting; prefix_project: default 2)")

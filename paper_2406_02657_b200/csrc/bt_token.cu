@@ -271,8 +271,14 @@ token_step_pipelined_kernel(TokenArgs a, int seqs_per_cta, int threads_per_seq)
     auto slot_addr = [&](int stage, int slot) -> uint32_t {
         return (uint32_t)__cvta_generic_to_shared(slots_mem + ((size_t)stage * n_slots + slot) * kTokThreads + tid);
     };
+    // Attend only (k_new == NULL: the step's row was cached by the projection that produced it): nothing is
+    // appended, the query sees all len rows, neither the cache nor the length is written.
+    const bool appended = a.k_new != nullptr;
     // rows of the cache this thread must fetch for a sequence whose length (before the step) is len
-    auto rows_to_read = [&](int len) -> int { return (len < 0 || len + 1 > a.cap) ? 0 : len; };
+    auto rows_to_read = [&](int len) -> int {
+        if (appended) return (len < 0 || len + 1 > a.cap) ? 0 : len;
+        return len < 0 ? 0 : (len > max_rows ? max_rows : len);   // the launcher guarantees cap <= max_rows here
+    };
     // the new row and the query do not depend on the length ...
     auto issue_new = [&](int i) {
         const int b = seq_of(i);
@@ -280,8 +286,10 @@ token_step_pipelined_kernel(TokenArgs a, int seqs_per_cta, int threads_per_seq)
             const int stage = i % kStages;
             const size_t slab = (size_t)b * a.H + h;
             cp_async16(slot_addr(stage, 0), reinterpret_cast<const bf16*>(a.q) + slab * HD + sub * 8);
-            cp_async16(slot_addr(stage, 1), reinterpret_cast<const bf16*>(a.k_new) + slab * HD + sub * 8);
-            cp_async16(slot_addr(stage, 2), reinterpret_cast<const bf16*>(a.v_new) + slab * HD + sub * 8);
+            if (appended) {
+                cp_async16(slot_addr(stage, 1), reinterpret_cast<const bf16*>(a.k_new) + slab * HD + sub * 8);
+                cp_async16(slot_addr(stage, 2), reinterpret_cast<const bf16*>(a.v_new) + slab * HD + sub * 8);
+            }
         }
     };
     // ... the cached rows to fetch do
@@ -315,8 +323,10 @@ token_step_pipelined_kernel(TokenArgs a, int seqs_per_cta, int threads_per_seq)
             const size_t slab = (size_t)b * a.H + h;
             if ((sub & 7) == 0) {  // one request per 128-byte line
                 prefetch_l2(reinterpret_cast<const bf16*>(a.q) + slab * HD + sub * 8);
-                prefetch_l2(reinterpret_cast<const bf16*>(a.k_new) + slab * HD + sub * 8);
-                prefetch_l2(reinterpret_cast<const bf16*>(a.v_new) + slab * HD + sub * 8);
+                if (appended) {
+                    prefetch_l2(reinterpret_cast<const bf16*>(a.k_new) + slab * HD + sub * 8);
+                    prefetch_l2(reinterpret_cast<const bf16*>(a.v_new) + slab * HD + sub * 8);
+                }
             }
             if (within == 0) prefetch_l2(a.len + b);
         }
@@ -343,15 +353,17 @@ token_step_pipelined_kernel(TokenArgs a, int seqs_per_cta, int threads_per_seq)
 
         const int b = seq_of(i);
         const int len_raw = lens[0];
-        const bool overflow = len_raw < 0 || len_raw + 1 > a.cap;
-        const int n_old = (b >= 0 && !overflow) ? len_raw : 0;
+        const bool overflow = appended && (len_raw < 0 || len_raw + 1 > a.cap);
+        const int n_old = (b >= 0 && !overflow) ? rows_to_read(len_raw) : 0;
         const int stage = i % kStages;
         const uint4* my = slots_mem + (size_t)stage * n_slots * kTokThreads + tid;
         uint4 qr = make_uint4(0, 0, 0, 0), kr = qr, vr = qr;
         if (b >= 0) {
             qr = my[0];
-            kr = my[kTokThreads];
-            vr = my[2 * kTokThreads];
+            if (appended) {
+                kr = my[kTokThreads];
+                vr = my[2 * kTokThreads];
+            }
         }
         float qf[8];
         unpack8(qr, qf);
@@ -377,7 +389,7 @@ token_step_pipelined_kernel(TokenArgs a, int seqs_per_cta, int threads_per_seq)
         }
         {
             const float d = row_sum<LPR>(TOK_DOT(kr));
-            sc[kMaxRows] = (b >= 0 && !overflow) ? d : kNegInf;
+            sc[kMaxRows] = (appended && b >= 0 && !overflow) ? d : kNegInf;
         }
 #undef TOK_DOT
         float mx = sc[kMaxRows];
@@ -412,7 +424,7 @@ token_step_pipelined_kernel(TokenArgs a, int seqs_per_cta, int threads_per_seq)
         }
         if (b >= 0) {
             const size_t slab = (size_t)b * a.H + h;
-            if (!overflow) {
+            if (appended && !overflow) {
                 bf16* cache = reinterpret_cast<bf16*>(a.kv) + slab * a.cap * 2 * HD + sub * 8;
                 *reinterpret_cast<uint4*>(cache + (size_t)len_raw * 2 * HD) = kr;
                 *reinterpret_cast<uint4*>(cache + (size_t)len_raw * 2 * HD + HD) = vr;
@@ -427,8 +439,10 @@ token_step_pipelined_kernel(TokenArgs a, int seqs_per_cta, int threads_per_seq)
         if (b >= 0 && within == 0) {
             if (overflow)
                 raise_status(a.dev_status, BT_DEV_OVERFLOW);
-            else
+            else if (appended)
                 a.len[b] = len_raw + 1;
+            else if (n_old == 0)
+                raise_status(a.dev_status, BT_DEV_EMPTY);   // a query with nothing to see: zeros out
         }
 #pragma unroll
         for (int d = 0; d + 1 < kLens; ++d) lens[d] = lens[d + 1];
@@ -466,17 +480,20 @@ cudaError_t launch_token_decode(const TokenArgs& a, cudaStream_t stream)
 {
     const int lpr = a.hd / 8;
     const int tps = a.H * lpr;  // threads per sequence (validated <= 256 by the caller)
-    if (a.n_q == 1 && a.k_new != nullptr && a.cap - 1 <= 12) {
+    // cached rows a step may have to read: all but the one being appended, or all of them when attending only
+    const int max_cached = a.k_new != nullptr ? a.cap - 1 : a.cap;
+    const bool attend_only_with_reset = a.k_new == nullptr && (a.reset_first || a.reset_mask != nullptr);   // general kernel
+    if (a.n_q == 1 && !attend_only_with_reset && max_cached <= 12) {
         // hot path: persistent pipelined kernel; deeper pipeline when the slots are small
         int spc_p = kTokThreads / tps;
         if (spc_p > a.B) spc_p = a.B;
-        if (a.cap - 1 <= 4)
+        if (max_cached <= 4)
             return a.hd == 64 ? launch_pipelined<64, BT_TOK_DEPTH4, 4, BT_TOK_CTAS4>(a, spc_p, tps, stream)
                               : launch_pipelined<128, BT_TOK_DEPTH4, 4, BT_TOK_CTAS4>(a, spc_p, tps, stream);
-        if (a.cap - 1 <= 5)  // e.g. L_B = 4 with the paper's main prefix length P = 2: still two CTAs per SM
+        if (max_cached <= 5)  // e.g. L_B = 4 with the paper's main prefix length P = 2: still two CTAs per SM
             return a.hd == 64 ? launch_pipelined<64, 1, 5, 2>(a, spc_p, tps, stream)
                               : launch_pipelined<128, 1, 5, 2>(a, spc_p, tps, stream);
-        if (a.cap - 1 > 8)  // the longest prefixes of the prefix-length ablation (P = 8 with L_B up to 5): 9 to 12 cached rows
+        if (max_cached > 8)  // the longest prefixes of the prefix-length ablation (P = 8 with L_B up to 5): 9 to 12 cached rows
             return a.hd == 64 ? launch_pipelined<64, 1, 12, 1>(a, spc_p, tps, stream)
                               : launch_pipelined<128, 1, 12, 1>(a, spc_p, tps, stream);
         // Deep local caches (6 to 8 cached rows).  A batch small enough for one wave of two CTAs per SM runs

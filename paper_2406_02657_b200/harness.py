@@ -451,3 +451,53 @@ class ProjectRun:
     def replay(self):
         """`sets` steps."""
         self.graph.replay()
+
+
+class ProjectedTokenRun:
+    """Token-decoder steps with the QKV projection in the path (sections 2.3 and 2.4 with the projections either
+    side): per layer and step, the layer's input x [B,1,D] is projected, the epilogue writes the K and V rows
+    into the local cache (reset at the first step of a block) and q goes to the attention call, which attends
+    over the cache as it stands (nothing left to append).  Two library calls per layer and step; distinct
+    weights per layer; step inputs rotate over a ring.  Prefix length 1: the block start is a one-row step too."""
+
+    def __init__(self, w, device="cuda", fill=None, ring=8):
+        assert w.prefix_len == 1
+        self.w, self.ring = w, ring
+        L, B, H, hd = w.n_layers, w.batch, w.heads, w.head_dim
+        D = H * hd
+        self.cfg = bt.make_config(B, H, hd, w.block_len, w.prefix_len, max(1, w.max_blocks), L)
+        mk = fill if fill is not None else (lambda tid, sh: torch.zeros(sh, dtype=torch.bfloat16, device=device))
+        self.cache = bt.LocalCache(self.cfg, device)
+        self.x = mk(50, (ring, L, B, 1, D))
+        self.x.mul_(1.0 / D ** 0.5)   # unit-variance q and k after the projection, as every attention input here
+        self.wt, self.bias = mk(51, (L, 3 * D, D)), mk(52, (L, 3 * D))
+        self.q = torch.empty((L, B, H, 1, hd), dtype=torch.bfloat16, device=device)
+        self.out = torch.empty((L, B, H, 1, hd), dtype=torch.bfloat16, device=device)
+        self.status = torch.zeros(1, dtype=torch.int32, device=device)
+        self.t = 0
+        self.launches_per_step = 3 * L   # product, length update, attention
+
+    def token_step(self):
+        w = self.w
+        first = self.t % w.block_len == 0
+        r = self.t % self.ring
+        for l in range(w.n_layers):
+            bt.bt_local_qkv_project_append(self.cfg, self.cache, l, self.x[r, l], self.wt[l], self.bias[l], self.q[l],
+                                           reset_first=first, dev_status=self.status)
+            bt.bt_token_decode_attn(self.cfg, self.cache, l, self.q[l], None, None, self.out[l], n_q=1, dev_status=self.status)
+        self.t += 1
+
+    def capture(self, n_steps=None):
+        n_steps = self.ring if n_steps is None else n_steps
+        assert n_steps % self.w.block_len == 0 and self.t % self.w.block_len == 0
+        for _ in range(self.w.block_len):
+            self.token_step()   # anything lazy happens outside the capture; a whole block keeps the phase
+        torch.cuda.synchronize()
+        self.graph = torch.cuda.CUDAGraph()
+        with torch.cuda.graph(self.graph):
+            for _ in range(n_steps):
+                self.token_step()
+        return n_steps
+
+    def replay(self):
+        self.graph.replay()

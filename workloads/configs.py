@@ -69,6 +69,8 @@ QKV_PROJECT_TOKEN = Workload("qkv_project_token", batch=4096, heads=16, head_dim
                              n_layers=12, max_blocks=1, seed=1033)
 QKV_PROJECT_BLOCK = Workload("qkv_project_block", batch=256, heads=16, head_dim=64, block_len=4, prefix_len=1,
                              n_layers=12, max_blocks=512, ctx_blocks=512, seed=1032)
+TOKEN_DECODE_PROJECTED = Workload("token_decode_projected", batch=4096, heads=16, head_dim=64, block_len=4, prefix_len=1,
+                                  n_layers=12, max_blocks=1, seed=1035)
 PREFIX_PROJECT = Workload("prefix_project", batch=4096, heads=16, head_dim=64, block_len=4, prefix_len=2,
                           n_layers=12, max_blocks=1, seed=1034)
 
@@ -88,4 +90,4 @@ def scaled(w: Workload, **kw) -> Workload:
 
 
 BY_NAME = {w.name: w for w in (TINY, BLOCK_DECODE, BLOCK_DECODE_16K, DENSE_DECODE, TOKEN_DECODE, BLOCK_PREFILL, BLOCK_PREFILL_8K,
-                               QKV_PROJECT_TOKEN, QKV_PROJECT_BLOCK, PREFIX_PROJECT)}
+                               QKV_PROJECT_TOKEN, QKV_PROJECT_BLOCK, PREFIX_PROJECT, TOKEN_DECODE_PROJECTED)}
