@@ -7,13 +7,14 @@
 //     local cache, so no separate append pass touches them.
 //
 // One persistent CTA per SM, warp-specialised:
-//   warps 0-3       : epilogue - thread = accumulator row (= tensor-memory lane).  64 columns at a time:
+//   warps 0-7       : epilogue - thread = accumulator row (= tensor-memory lane), two warps per lane quarter
+//                     taking alternate 64-column pieces.  64 columns at a time:
 //                     tensor memory -> registers, + bias, -> bf16, through a per-warp swizzled
 //                     shared-memory patch so that the global stores are whole 128-byte lines (8 lanes
 //                     per row piece: one head of one cache row at head_dim 64), then to q / the cache /
 //                     the plain [M][N] output
-//   warp 4 (1 lane) : TMA producer - x tile [128 x 64] and W tile [BN x 64] per stage, 128-byte swizzle
-//   warp 5 (1 lane) : tcgen05.mma issuer - 128 x BN x 16 instructions, fp32 accumulators in tensor
+//   warp 8 (1 lane) : TMA producer - x tile [128 x 64] and W tile [BN x 64] per stage, 128-byte swizzle
+//   warp 9 (1 lane) : tcgen05.mma issuer - 128 x BN x 16 instructions, fp32 accumulators in tensor
 //                     memory, double-buffered so that the epilogue of a tile runs under the next
 //                     tile's products
 // BN (64, 128 or 256 output features per tile) is chosen per launch so that there are enough tiles
@@ -42,8 +43,8 @@ using namespace tc;
 
 constexpr int BM = 128;                  // rows of x per tile (= tensor-memory lanes)
 constexpr int BK = 64;                   // K elements per stage: one 128-byte swizzle atom
-constexpr int kEpilogueWarps = 4, kProducerWarp = 4, kMmaWarp = 5;
-constexpr int kThreads = 192;
+constexpr int kEpilogueWarps = 8, kProducerWarp = 8, kMmaWarp = 9;
+constexpr int kThreads = 320;
 constexpr uint32_t kABytes = BM * BK * 2;
 constexpr uint32_t kSpinLimit = 1u << 26;
 constexpr uint64_t kWaitLimitNs = 1000000000ull;  // 1 s: far beyond any legitimate wait
@@ -273,9 +274,11 @@ project_tc_kernel(const __grid_constant__ CUtensorMap mapX, const __grid_constan
         }
     } else {
         // ------------------------------------------------------------------ epilogue: thread = output row
-        const int wq = warp;                                   // warps 0-3: tensor-memory lane quarter
+        // warps 0-7: warp e drains tensor-memory lane quarter e % 4 (the quarter a warp may access is its index
+        // modulo 4) and every other 64-column piece, starting at piece e / 4
+        const int wq = warp & 3, half = warp >> 2;
         const uint32_t lane_base = tmem + ((uint32_t)(wq * 32) << 16);
-        const uint32_t patch = sPatch + wq * kPatchBytes;
+        const uint32_t patch = sPatch + warp * kPatchBytes;
         const bf16* bias = reinterpret_cast<const bf16*>(a.bias);
         const int D = a.H * a.hd;
         uint32_t t = 0;
@@ -303,7 +306,7 @@ project_tc_kernel(const __grid_constant__ CUtensorMap mapX, const __grid_constan
             if (!ok) break;
             tc_fence_after();
 #pragma unroll 1
-            for (int c0 = 0; c0 < BN; c0 += 64) {
+            for (int c0 = half * 64; c0 < BN; c0 += 128) {
                 const int col0 = tn * BN + c0;                 // first output feature of this 64-column piece
                 if (col0 >= a.N) break;                        // warp-uniform
                 uint32_t r[64];
