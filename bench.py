@@ -422,6 +422,19 @@ def measure(name, w, args, env, primary):
                             ms / n_layer_steps, n_layer_steps * alg, ms, None)
         add_tensor_roofline(roof, pk, fl, alg, ms / n_layer_steps, in_long_step=False)
         launches = run.launches_per_step * n_tok * steps
+        if not args.no_cpu_baseline:
+            import oracle
+            n_seq, n_st = 32, w.block_len
+            oc = oracle.Cache(n_seq, w.heads, w.local_cap, w.head_dim)
+            xs = [gen.normal_bf16_bits(w.seed, 60 + t, (n_seq, 1, D)) for t in range(n_st)]
+            Wq, bq = gen.normal_bf16_bits(w.seed, 70, (3 * D, D)), gen.normal_bf16_bits(w.seed, 71, (3 * D,))
+
+            def go():
+                for t in range(n_st):
+                    q = oracle.qkv_project_append(oc, xs[t], Wq, bq, reset_first=(t == 0))
+                    oracle.token_decode_attn(oc, oracle.round_to_bf16(q), None, None)
+            cpu = oracle_sample(go, n_seq * n_st / w.n_layers, f"{n_seq} of {w.batch} sequences x 1 of {w.n_layers} layers x {n_st} token steps "
+                                                              f"(projection + append + attention, fp64)")
     elif name == "sweep":
         # a step = one whole generation: prompt prefill + bulk append, then gen_tokens / L_B generated blocks
         # (CUDA-graph replays of `ring` blocks each); tokens = batch x generated tokens
