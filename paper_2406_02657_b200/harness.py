@@ -198,12 +198,10 @@ class DenseDecodeStep:
         torch.cuda.synchronize()
         self.graph = torch.cuda.CUDAGraph()
         with torch.cuda.graph(self.graph):
-            for s in range(self.sets):
-                self.rewind()
-                self.step(s)
+            self.rewind()
+            self.step()
 
     def replay(self):
-        """`sets` steps."""
         self.graph.replay()
 
 
