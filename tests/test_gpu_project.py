@@ -259,3 +259,30 @@ def test_qkv_projection_at_the_bench_shapes(bt, B, H, hd, n):
     for g, r in ((gk, oc.k), (gv, oc.v)):
         err = np.abs(widen(g) - widen(r))
         assert (err <= 2e-3 + 8e-3 * np.abs(widen(r))).all()      # rows outside the window are zero on both sides
+
+
+# ------------------------------------------------------------------ the prompt's path with the projection in
+
+@pytest.mark.parametrize("hd,T", [(64, 200), (128, 130)])
+def test_prompt_projection_then_prefill_from_the_cache(bt, hd, T):
+    """The block decoder's prefill with the projection in front (sections 2.1, 2.3): the prompt's T block embeddings
+    are projected in one call, the epilogue writes the T K,V rows of every sequence into the block cache, and the
+    prefill attention reads K and V in place from the cache.  Against the oracle's projection + append + dense
+    causal attention; lengths exact."""
+    B, H, N = 3, 4, 256
+    D = H * hd
+    cfg = bt.make_config(B, H, hd, 4, 1, N, 1)
+    cache = bt.BlockCache(cfg)
+    x = unit_rows(780 + hd, 0, (B, T, D))
+    W, bias = rnd(780 + hd, 1, (3 * D, D)), rnd(780 + hd, 2, (3 * D,))
+    q = torch.empty((B, H, T, hd), dtype=torch.bfloat16, device="cuda")
+    out = torch.empty((B, H, T, hd), dtype=torch.bfloat16, device="cuda")
+    st = status_word()
+    bt.bt_block_qkv_project_append(cfg, cache, 0, to_dev(x), to_dev(W), to_dev(bias), q, dev_status=st)
+    bt.bt_block_prefill_attn(cfg, q, cache.k[0], cache.v[0], out, n_blocks=T, kv_seq_stride=N, dev_status=st)
+    oc = oracle.Cache(B, H, N, hd)
+    q_ref = oracle.qkv_project_append(oc, x, W, bias)
+    assert_close_proj(q, q_ref, "q of the prompt projection")
+    assert cache.len[0].cpu().tolist() == oc.len.tolist() == [T] * B and st.item() == 0
+    ref = oracle.block_prefill_attn(oracle.round_to_bf16(q_ref), oc.k, oc.v, kv_seq_stride=N)
+    assert_close(out, ref, "prefill attention over the projected cache", p_bf16=True)
