@@ -58,24 +58,6 @@ __device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatil
 
 using namespace tc;
 
-__device__ __forceinline__ bool elect_one()
-{
-    uint32_t pred;
-    asm volatile("{\n\t.reg .pred P;\n\telect.sync _|P, 0xffffffff;\n\tselp.u32 %0, 1, 0, P;\n\t}" : "=r"(pred));
-    return pred != 0;
-}
-
-// A shared-memory matrix descriptor from its two halves (see make_desc: bits 0-13 address / 16, bits 16-29 leading
-// dimension / 16 in the low word; bits 32-45 stride / 16, bit 46 the version, bits 61-63 the swizzle in the high word).
-// The high word (8-row group pitch 1024 bytes, version, 128-byte swizzle) is the same for every operand here.
-constexpr uint32_t kDescHi = (1024u >> 4) | (1u << 14) | (2u << 29);
-__device__ __forceinline__ uint64_t desc_words(uint32_t lo, uint32_t hi)
-{
-    uint64_t d;
-    asm("mov.b64 %0, {%1, %2};" : "=l"(d) : "r"(lo), "r"(hi));
-    return d;
-}
-
 __device__ __forceinline__ float ex2(float x)
 {
     float y;
@@ -152,11 +134,9 @@ struct Schedule {
 enum {
     B_QFULL = 0,                       // [kQBufs]  TMA -> MMA
     B_QEMPTY = B_QFULL + kQBufs,       // [kQBufs]  epilogue (output staged in the buffer has been read by its store) -> TMA
-    B_KFULL = B_QEMPTY + kQBufs,       // [kKvStages]
-    B_KEMPTY = B_KFULL + kKvStages,
-    B_VFULL = B_KEMPTY + kKvStages,
-    B_VEMPTY = B_VFULL + kKvStages,
-    B_SFULL = B_VEMPTY + kKvStages,    // [2 tiles][2 buffers]: S ready
+    B_KFULL = B_QEMPTY + kQBufs,       // [kKvStages]  K_j and V_j of a stage have both landed
+    B_KEMPTY = B_KFULL + kKvStages,    // [kKvStages]  both tiles' P V products on the stage are done (two arrivals)
+    B_SFULL = B_KEMPTY + kKvStages,    // [2 tiles][2 buffers]: S ready
     B_PFULL = B_SFULL + 4,             // [2 tiles][2 buffers]: 128 softmax threads have written P over it
     B_PVDONE = B_PFULL + 4,            // [2 tiles]: one completion per P V product (O may be rescaled after it)
     B_OFULL = B_PVDONE + 2,            // [2 tiles]: last P V of the item done
@@ -226,7 +206,7 @@ block_prefill_tc_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_c
 
     if (threadIdx.x == 0) {
         for (int i = 0; i < B_COUNT; ++i)
-            mbar_init(bar(i), (i >= B_PFULL && i < B_PFULL + 4) ? 128u : (i >= B_KEMPTY && i < B_KEMPTY + kKvStages) || (i >= B_VEMPTY && i < B_VEMPTY + kKvStages) ? 2u : 1u);
+            mbar_init(bar(i), (i >= B_PFULL && i < B_PFULL + 4) ? 128u : (i >= B_KEMPTY && i < B_KEMPTY + kKvStages) ? 2u : 1u);
         *abort_flag = 0;
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     }
@@ -287,14 +267,11 @@ block_prefill_tc_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_c
                     const uint32_t st = kv_count % kKvStages, par = ((kv_count / kKvStages) & 1) ^ 1;
                     ok = ok && mbar_wait(bar(B_KEMPTY + st), par, abort_flag, p.dev_status);
                     if (!ok) return;
-                    mbar_expect_tx(bar(B_KFULL + st), KV_TILE_BYTES);
+                    mbar_expect_tx(bar(B_KFULL + st), 2 * KV_TILE_BYTES);  // K and V of a stage arrive on one barrier
                     for (int bx = 0; bx < NB; ++bx)
                         tma_load_3d(sK + st * KV_TILE_BYTES + bx * kKvBoxBytes, &mapK, bar(B_KFULL + st), bx * 64, j * BN, it.bh);
-                    ok = mbar_wait(bar(B_VEMPTY + st), par, abort_flag, p.dev_status);
-                    if (!ok) return;
-                    mbar_expect_tx(bar(B_VFULL + st), KV_TILE_BYTES);
                     for (int bx = 0; bx < NB; ++bx)
-                        tma_load_3d(sV + st * KV_TILE_BYTES + bx * kKvBoxBytes, &mapV, bar(B_VFULL + st), bx * 64, j * BN, it.bh);
+                        tma_load_3d(sV + st * KV_TILE_BYTES + bx * kKvBoxBytes, &mapV, bar(B_KFULL + st), bx * 64, j * BN, it.bh);
                     ++kv_count;
                 };
                 // Q_A and the first two key/value tiles come first (tile A's first two products need just these);
@@ -353,18 +330,15 @@ block_prefill_tc_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_c
                         for (int kk = 0; kk < HD / 16; ++kk) {
                             const uint32_t qoff = (uint32_t)(((kk >> 2) * kQBoxBytes + (kk & 3) * 32) >> 4);
                             const uint32_t koff = (uint32_t)(((kk >> 2) * kKvBoxBytes + (kk & 3) * 32) >> 4);
-                            mma_bf16(d_s, desc_words(qlo + qoff, kDescHi), desc_words(klo + koff, kDescHi), IDESC_S, kk > 0 ? 1u : 0u);
+                            mma_bf16(d_s, desc_words(qlo + qoff, kDescHiSw128), desc_words(klo + koff, kDescHiSw128), IDESC_S, kk > 0 ? 1u : 0u);
                         }
                         mma_commit(bar(B_SFULL + x * 2 + (j & 1)));
-                        mma_commit(bar(B_KEMPTY + st));
-                        if (x == 0 && j >= it.nb) mma_commit(bar(B_KEMPTY + st));  // tile B does not read this one
                     }
                     __syncwarp();
                 };
                 // O_x (+)= P_x(j) V_j
                 auto issue_pv = [&](int j) {
                     const uint32_t kc = kv_base + j, st = kc % kKvStages;
-                    ok = ok && wait_all(bar(B_VFULL + st), (kc / kKvStages) & 1);
                     ok = ok && wait_all(bar(B_PFULL + x * 2 + (p_count & 1)), (p_count >> 1) & 1);
                     if (!ok) return;
                     ++p_count;
@@ -376,11 +350,12 @@ block_prefill_tc_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_c
                     if (elect_one()) {
 #pragma unroll
                         for (int kk = 0; kk < BN / 16; ++kk)
-                            mma_bf16_ts(tmem + COL_O0 + x * HD, a_p + kk * 8, desc_words(vlo + (uint32_t)kk * 128u, kDescHi), IDESC_O,
+                            mma_bf16_ts(tmem + COL_O0 + x * HD, a_p + kk * 8, desc_words(vlo + (uint32_t)kk * 128u, kDescHiSw128), IDESC_O,
                                         (j > 0 || kk > 0) ? 1u : 0u);
                         mma_commit(bar(B_PVDONE + x));
-                        mma_commit(bar(B_VEMPTY + st));
-                        if (x == 0 && j >= it.nb) mma_commit(bar(B_VEMPTY + st));  // tile B does not read this one
+                        // the stage (K_j and V_j) is free after its last reader
+                        mma_commit(bar(B_KEMPTY + st));
+                        if (x == 0 && j >= it.nb) mma_commit(bar(B_KEMPTY + st));  // tile B does not read this one
                         if (j == steps - 1) mma_commit(bar(B_OFULL + x));
                     }
                     __syncwarp();

@@ -240,35 +240,44 @@ project_tc_kernel(const __grid_constant__ CUtensorMap mapX, const __grid_constan
             }
         }
     } else if (warp == kMmaWarp) {
-        if (lane == 0 && leader) {   // a pair's products are issued by its leader alone
+        // The whole warp walks the loop (control flow stays warp-uniform; the outcome of every wait is agreed on by
+        // a vote) and one elected lane issues: a lone lane inside a divergent branch issues tcgen05.mma slower.
+        if (leader) {   // a pair's products are issued by its leader alone
+            auto wait_all = [&](uint32_t b, uint32_t parity) { return __all_sync(0xffffffffu, wait(b, parity, abort_flag, a.dev_status)) != 0; };
             uint32_t it = 0, t = 0;
             bool ok = true;
             for (int tile = unit; ok && tile < n_tiles; tile += n_units, ++t) {
                 const uint32_t acc = t & 1;
-                ok = wait(acc_empty(acc), ((t >> 1) & 1) ^ 1, abort_flag, a.dev_status);  // the epilogue has drained this accumulator
+                ok = wait_all(acc_empty(acc), ((t >> 1) & 1) ^ 1);  // the epilogue has drained this accumulator
                 if (!ok) break;
                 tc_fence_after();
                 for (int kb = 0; kb < n_kb; ++kb, ++it) {
                     const uint32_t s = it % S;
-                    ok = wait(full(s), (it / S) & 1, abort_flag, a.dev_status);
+                    ok = wait_all(full(s), (it / S) & 1);
                     if (!ok) break;
                     tc_fence_after();
+                    // descriptor low words: address in 16-byte units plus the leading-dimension field; 16 elements
+                    // of K are 32 bytes inside a swizzled 128-byte row
                     const uint32_t a0 = base + s * C::kStageBytes, b0 = a0 + kABytes;
+                    const uint32_t alo = (a0 >> 4) | (1u << 16), blo = (b0 >> 4) | (1u << 16);
+                    if (elect_one()) {
 #pragma unroll
-                    for (int kk = 0; kk < BK / 16; ++kk) {
-                        if constexpr (kCtas == 1)
-                            mma_bf16(tmem + acc * BN, make_desc(a0 + kk * 32, 16, 1024), make_desc(b0 + kk * 32, 16, 1024), IDESC,
-                                     (kb > 0 || kk > 0) ? 1u : 0u);
-                        else
-                            mma_bf16_pair(tmem + acc * BN, make_desc(a0 + kk * 32, 16, 1024), make_desc(b0 + kk * 32, 16, 1024), IDESC,
-                                          (kb > 0 || kk > 0) ? 1u : 0u);
+                        for (int kk = 0; kk < BK / 16; ++kk) {
+                            if constexpr (kCtas == 1)
+                                mma_bf16(tmem + acc * BN, desc_words(alo + kk * 2, kDescHiSw128), desc_words(blo + kk * 2, kDescHiSw128), IDESC,
+                                         (kb > 0 || kk > 0) ? 1u : 0u);
+                            else
+                                mma_bf16_pair(tmem + acc * BN, desc_words(alo + kk * 2, kDescHiSw128), desc_words(blo + kk * 2, kDescHiSw128), IDESC,
+                                              (kb > 0 || kk > 0) ? 1u : 0u);
+                        }
+                        if constexpr (kCtas == 1) mma_commit(empty(s));
+                        else mma_commit_pair(empty(s));
+                        if (kb == n_kb - 1) {
+                            if constexpr (kCtas == 1) mma_commit(acc_full(acc));
+                            else mma_commit_pair(acc_full(acc));
+                        }
                     }
-                    if constexpr (kCtas == 1) mma_commit(empty(s));
-                    else mma_commit_pair(empty(s));
-                }
-                if (ok) {
-                    if constexpr (kCtas == 1) mma_commit(acc_full(acc));
-                    else mma_commit_pair(acc_full(acc));
+                    __syncwarp();
                 }
             }
         }

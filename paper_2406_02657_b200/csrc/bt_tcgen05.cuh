@@ -42,6 +42,26 @@ __device__ __forceinline__ uint64_t make_desc(uint32_t saddr, uint32_t lbo_bytes
     return d;
 }
 
+// The same descriptor from its two 32-bit halves.  For the operands used here (8-row groups 1024 bytes apart, 128-byte
+// swizzle) the high word is a constant and the low word is the start address in 16-byte units plus the
+// leading-dimension field, so stepping through a tile costs one add per instruction.
+constexpr uint32_t kDescHiSw128 = (1024u >> 4) | (1u << 14) | (2u << 29);
+__device__ __forceinline__ uint64_t desc_words(uint32_t lo, uint32_t hi)
+{
+    uint64_t d;
+    asm("mov.b64 %0, {%1, %2};" : "=l"(d) : "r"(lo), "r"(hi));
+    return d;
+}
+
+// One lane of a converged warp.  tcgen05.mma issued under this predicate, in a loop that the whole warp walks,
+// keeps the pace of the tensor pipe; issued by lane 0 inside a divergent branch it does not.
+__device__ __forceinline__ bool elect_one()
+{
+    uint32_t pred;
+    asm volatile("{\n\t.reg .pred P;\n\telect.sync _|P, 0xffffffff;\n\tselp.u32 %0, 1, 0, P;\n\t}" : "=r"(pred));
+    return pred != 0;
+}
+
 // Instruction descriptor: bf16 x bf16 -> fp32, A K-major, B K-major or MN-major.
 __host__ __device__ constexpr uint32_t make_idesc(int M, int N, bool b_mn_major)
 {
