@@ -220,3 +220,20 @@ def test_block_prefill_8k_prompt_full_size(bt):
         q, k, v = (gen.torch_to_bits(x[l, b:b + 1, h:h + 1]) for x in (run.q, run.k, run.v))
         ref = oracle.block_prefill_attn(q, k, v)
         assert_close(run.out[l, b:b + 1, h:h + 1], ref, f"8K-prompt prefill layer {l} b {b} h {h}", p_bf16=True)
+
+
+def test_block_prefill_many_items_ragged_last_tile(bt):
+    """A launch too large for the host-made item table (768 (sequence, head) pairs x 7 pairs of query tiles), so
+    the CTAs walk the items round robin, with a prompt that ends half way into its last query tile (1600 blocks =
+    12.5 tiles): every row written, sampled (sequence, head) pairs against the oracle."""
+    from paper_2406_02657_b200 import harness
+    w = configs.scaled(configs.BLOCK_PREFILL, batch=48, prompt_blocks=1600, max_blocks=1600, n_layers=1)
+    run = harness.PrefillRun(w, fill=_fill(w))
+    run.out.fill_(float("nan"))
+    run.step()
+    torch.cuda.synchronize()
+    assert torch.isfinite(run.out.float()).all()
+    for l, b, h in ((0, 0, 0), (0, 47, 15), (0, 23, 9)):
+        q, k, v = (gen.torch_to_bits(x[l, b:b + 1, h:h + 1]) for x in (run.q, run.k, run.v))
+        ref = oracle.block_prefill_attn(q, k, v)
+        assert_close(run.out[l, b:b + 1, h:h + 1], ref, f"many-item prefill b {b} h {h}", p_bf16=True)
