@@ -242,7 +242,8 @@ NCU_TRAFFIC_BYTES = {
     # reads equal the algorithmic reads; the 25.2 MB written per launch mostly reach DRAM after the launch and
     # are counted at their algorithmic size
     ("token_decode", 1): 75.5e6,
-    ("block_prefill", 1): 220.4e6,     # 110.2 MB captured at batch 16 (reads exact; 9.4 of 33.5 MB of writes reach DRAM inside the launch)
+    ("block_prefill", 1): 220.4e6,     # 110.2 MB captured at batch 16 (reads exact; 9-10 of 33.5 MB of writes reach DRAM inside the launch)
+    ("block_prefill_8k", 1): 262.6e6,  # captured at full size: 216-218 MB read (Q, K, V are 201 MB), 45.5-46.5 of 67 MB written inside the launch
     # reads are x and W exactly once (14.7 MB); the 25.2 MB of q, K, V rows written stay in L2 until after the launch
     # and are counted at their algorithmic size
     ("qkv_project_token", 1): 39.9e6,
@@ -504,7 +505,7 @@ def measure(name, w, args, env, primary):
         alg = traffic.prefill_layer_bytes(w.batch, w.heads, w.prompt_blocks, w.head_dim)
         fl = traffic.prefill_layer_flops(w.batch, w.heads, w.prompt_blocks, w.head_dim)
         roof = hbm_roofline(pk, "block_prefill_tc_kernel", alg, ms / w.n_layers, w.n_layers * alg, ms,
-                            NCU_TRAFFIC_BYTES.get((name, 1)) if w.batch == 32 else None)
+                            NCU_TRAFFIC_BYTES.get((name, 1)) if w.batch == configs.BY_NAME[name].batch else None)
         add_tensor_roofline(roof, pk, fl, alg, ms / w.n_layers, in_long_step=True)
         launches = run.launches_per_step * steps
         if not primary and not args.no_cpu_baseline:
